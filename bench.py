@@ -1,0 +1,529 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-branch-attention hot path (forward + backward).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one synthetic batch: metadata
+plan reuse, fused forward (through the partial-(O, LSE) + lse_merge zigzag
+path for the long-context workload), backward preprocess, dQ, dK/dV, gradient
+finalisation.  Prints ONE JSON line (rank 0).  `--impl reference` times the
+fp64 CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_07108_b200 import workloads as W  # noqa: E402
+
+METRIC = "branch_attn_fwd_bwd_useful_tflops"
+UNIT = "TFLOP/s"
+DATASHEET_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# name -> (config number, shrink, zigzag cp or 0, backward?)
+WORKLOADS = {
+    "config5_256k_zigzag": (5, 1, 8, True),
+    "config5_256k_monolithic": (5, 1, 0, True),
+    "config5_64k_zigzag": (5, 4, 8, True),
+    "config4_tree_64k": (4, 1, 0, True),
+    "config3_dflash_32k": (3, 1, 0, True),
+    "config2_eagle3_8k": (2, 1, 0, False),
+}
+
+
+def useful_flops(p, backward=True):
+    pairs = W.useful_pairs(p)
+    per_pair = 4 * p.head_dim * p.h_q
+    return pairs * per_pair * (3.5 if backward else 1.0), pairs
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# ----------------------------------------------------------------------------
+# distributed plumbing (replicas only: no data-path collective)
+# ----------------------------------------------------------------------------
+
+def dist_setup(n_gpus, backend=None):
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world <= 1:
+        return None, 0, 1
+    backend = backend or ("nccl" if torch.cuda.is_available() else "gloo")
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    dist.init_process_group(backend=backend)
+    return dist, dist.get_rank(), dist.get_world_size()
+
+
+def max_over_ranks(dist, value, device="cpu"):
+    """Slowest rank's time (the job finishes when the last replica does)."""
+    import torch
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(dist, flops_per_rank, local_ms, device="cpu"):
+    """Whole-job throughput: every rank processed `flops_per_rank`; time = max."""
+    world = 1 if dist is None else dist.get_world_size()
+    ms = max_over_ranks(dist, local_ms, device)
+    return world * flops_per_rank / (ms * 1e-3) / 1e12, ms
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "200", "-i", str(self.index)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, reasons, mx, power = [], set(), None, []
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx = float(f[2]); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                  "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            res.update(sm_mhz=statistics.median(sm), sm_max_mhz=mx, reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return res
+
+
+# ----------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------
+
+class Recorder:
+    """Wraps the binding: counts kernel launches and brackets each library call
+    with CUDA events on the launching stream so that per-kernel time inside the
+    timed region can be summed afterwards."""
+
+    def __init__(self, ba, plan_problem):
+        import torch
+        self.ba = ba
+        self.torch = torch
+        self.p = plan_problem
+        self.events = []           # (kind, start, end)
+        self.launches = 0
+        self.enabled = False
+        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL"):
+            setattr(self, name, getattr(ba, name))
+
+    def _wrap(self, kind, n_launch, fn, *a, **k):
+        if self.enabled:
+            s = self.torch.cuda.Event(enable_timing=True)
+            e = self.torch.cuda.Event(enable_timing=True)
+            s.record()
+            out = fn(*a, **k)
+            e.record()
+            self.events.append((kind, s, e))
+            self.launches += n_launch
+            return out
+        return fn(*a, **k)
+
+    def branch_attn_fwd(self, *a, **k):
+        return self._wrap("fwd", 1, self.ba.branch_attn_fwd, *a, **k)
+
+    def branch_attn_fwd_partial(self, *a, **k):
+        return self._wrap("fwd", 1, self.ba.branch_attn_fwd_partial, *a, **k)
+
+    def lse_merge(self, *a, **k):
+        return self._wrap("lse_merge", 1, self.ba.lse_merge, *a, **k)
+
+    def branch_attn_bwd(self, plan, q_main, *a, **k):
+        # delta (main rows, branch rows) + dQ + dK/dV
+        return self._wrap("bwd", 4 if q_main is not None else 3, self.ba.branch_attn_bwd, plan, q_main, *a, **k)
+
+    def ba_finalize_grads(self, *a, **k):
+        return self._wrap("finalize", 1, self.ba.ba_finalize_grads, *a, **k)
+
+    def totals(self):
+        out = {}
+        for kind, s, e in self.events:
+            out.setdefault(kind, [0.0, 0])
+            out[kind][0] += s.elapsed_time(e)
+            out[kind][1] += 1
+        return out
+
+
+def make_device_inputs(p, torch, device, seed=0):
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    dt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
+
+    def draw(shape, std):
+        return (torch.randn(shape, generator=g, device=device, dtype=torch.float32) * std).to(dt)
+
+    n, m = p.n_main, p.n_branch
+    t = {"q_main": draw((n, p.h_q, p.head_dim), 0.5), "q_branch": draw((m, p.h_q, p.head_dim), 0.5),
+         "k": draw((n + m, p.h_kv, p.head_dim), 0.5), "v": draw((n + m, p.h_kv, p.head_dim), 0.5),
+         "d_o": draw((n + m, p.h_q, p.head_dim), 0.1)}
+    return t
+
+
+def run_step(rec, plan, t, cp, backward):
+    from paper_2609_07108_b200 import zigzag
+    if cp:
+        o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp,
+                                   out=t.get("_o"), lse=t.get("_lse"))
+        grads = zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp) \
+            if backward else None
+    else:
+        o, lse = rec.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"],
+                                     out=t.get("_o"), lse=t.get("_lse"))
+        grads = rec.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"],
+                                    grads=t.get("_grads")) if backward else None
+    return o, lse, grads
+
+
+def run_ours(args):
+    import torch
+    from paper_2609_07108_b200 import binding as ba
+
+    dist, rank, world = dist_setup(args.gpus)
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+
+    name = args.workload
+    if name == "auto":
+        name = "config5_256k_zigzag"
+    cfg, shrink, cp, backward = WORKLOADS[name]
+    p = W.CONFIGS[cfg](shrink) if cfg != 1 else W.config1()
+    impl = {"auto": ba.IMPL_AUTO, "simt": ba.IMPL_SIMT, "tc": ba.IMPL_TC}[args.kernels]
+    plan = ba.Plan(p, device=device, impl=impl)
+    flops, pairs = useful_flops(p, backward)
+    t = make_device_inputs(p, torch, device)
+    if not cp:
+        t["_o"] = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
+        t["_lse"] = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=device)
+    rec = Recorder(ba, p)
+    in_bytes = sum(t[k].numel() * t[k].element_size() for k in ("q_main", "q_branch", "k", "v", "d_o"))
+    flush = None
+    if in_bytes < 512 << 20:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        run_step(rec, plan, t, cp, backward)
+        if flush is not None:
+            flush.fill_(1)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    rec.enabled = True
+    step_ms = []
+    barrier()
+    for _ in range(args.steps):
+        if flush is not None:
+            flush.fill_(1)
+        s = torch.cuda.Event(enable_timing=True)
+        e = torch.cuda.Event(enable_timing=True)
+        s.record()
+        run_step(rec, plan, t, cp, backward)
+        e.record()
+        step_ms.append((s, e))
+    barrier()
+    rec.enabled = False
+    clocks = sampler.stop() if rank == 0 else {}
+    local_ms = sum(s.elapsed_time(e) for s, e in step_ms)
+    value, total_ms = aggregate_throughput(dist, flops * args.steps, local_ms, device)
+    totals = rec.totals()
+    launches = rec.launches
+
+    # ---- end to end through the API with HOST buffers (pinned), copies timed
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args)
+
+    # ---- dominant kernel and its roofline
+    peaks = load_peaks()
+    roof = None
+    if totals:
+        kind = max(totals, key=lambda k: totals[k][0])
+        ms, calls = totals[kind]
+        # algorithmic flop of all launches of that kind over the timed steps
+        share = {"fwd": 4.0, "bwd": 10.0}.get(kind)
+        if share is not None:
+            kflops = pairs * p.head_dim * p.h_q * share * args.steps
+            achieved = kflops / (ms * 1e-3) / 1e12
+            long_step = total_ms / args.steps > 1000.0
+            peak = peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"]
+            roof = {"bound": "tensor", "kernel": kind, "achieved": round(achieved, 2), "peak": peak,
+                    "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": None,
+                    "peak_source": f"{peaks['_source']} {'sustained' if long_step else 'burst'} bf16",
+                    "launches": calls, "avg_launch_ms": round(ms / calls, 4),
+                    "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
+                    "frac_of_datasheet": round(achieved / DATASHEET_BF16_TFLOPS, 4)}
+        else:
+            roof = {"bound": "hbm", "kernel": kind, "achieved": None, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": None, "traffic": None}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(p, seconds_target=15.0)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(total_ms / args.steps, 3), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": p.dtype, "data": "synthetic",
+            "config": {"workload": name, "n_main": p.n_main, "rows": p.rows, "h_q": p.h_q, "h_kv": p.h_kv,
+                       "head_dim": p.head_dim, "mask": W.KIND_NAMES[p.kind], "pairs_per_head": pairs,
+                       "path": (f"zigzag cp={cp}: partial fwd + lse_merge, partial bwd accumulate"
+                                if cp else "monolithic fwd + bwd"),
+                       "backward": backward, "kernels": {ba.IMPL_SIMT: "simt", ba.IMPL_TC: "tcgen05"}[plan.impl],
+                       "l2": "inputs larger than L2" if flush is None else "256 MiB flush between steps",
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "frac_of_peak": {"burst": round(value / world / peaks["bf16_tflops"], 4),
+                             "sustained": round(value / world / peaks["bf16_tflops_sustained"], 4),
+                             "datasheet": round(value / world / DATASHEET_BF16_TFLOPS, 4),
+                             "source": peaks["_source"]},
+            "kernel_ms": {k: round(v[0] / args.steps, 3) for k, v in totals.items()},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "e2e": e2e,
+            "roofline": roof,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
+    """Same step, inputs in pinned host memory: H2D of Q/K/V/dO, the library
+    calls, D2H of O/LSE and the gradients, all inside the timed region."""
+    import psutil
+    names = ("q_main", "q_branch", "k", "v") + (("d_o",) if backward else ())
+    h2d = sum(t[k].numel() * t[k].element_size() for k in names)
+    out_shapes = [((p.rows, p.h_q, p.head_dim), plan.torch_dtype), ((p.rows, p.h_q), torch.float32)]
+    if backward:
+        out_shapes += [((p.n_main, p.h_q, p.head_dim), plan.torch_dtype),
+                       ((p.n_branch, p.h_q, p.head_dim), plan.torch_dtype),
+                       ((p.rows, p.h_kv, p.head_dim), plan.torch_dtype),
+                       ((p.rows, p.h_kv, p.head_dim), plan.torch_dtype)]
+    d2h = sum(int(np.prod(s)) * torch.empty(0, dtype=d).element_size() for s, d in out_shapes)
+    pin = psutil.virtual_memory().available > 3 * (h2d + d2h)
+    host_in = {}
+    for k in names:
+        host_in[k] = torch.empty(t[k].shape, dtype=t[k].dtype, pin_memory=pin)
+        host_in[k].copy_(t[k])
+    host_out = [torch.empty(s, dtype=d, pin_memory=pin) for s, d in out_shapes]
+    rec = Recorder(ba, p)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    steps = max(1, min(args.steps, args.e2e_steps))
+    s_ev = torch.cuda.Event(enable_timing=True)
+    e_ev = torch.cuda.Event(enable_timing=True)
+    s_ev.record()
+    for _ in range(steps):
+        for k in names:
+            t[k].copy_(host_in[k], non_blocking=True)
+        o, lse, grads = run_step(rec, plan, t, cp, backward)
+        outs = [o, lse] + (list(grads[:4]) if backward else [])
+        for dst, src in zip(host_out, outs):
+            dst.copy_(src, non_blocking=True)
+    e_ev.record()
+    torch.cuda.synchronize()
+    ms = s_ev.elapsed_time(e_ev)
+    value, _ = aggregate_throughput(dist, flops * steps, ms, device)
+    return {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "steps": steps, "ms_per_step": round(ms / steps, 3), "pinned": bool(pin)}
+
+
+# ----------------------------------------------------------------------------
+# CPU baseline = the oracle, as it stands, on a bounded sample
+# ----------------------------------------------------------------------------
+
+def oracle_sample(p, n_rows, seed=0):
+    """Rows sampled uniformly from the workload (main and branch rows), one KV
+    group (h_q/h_kv query heads).  Returns the inputs and the sampled pairs."""
+    import copy
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(p.rows, size=min(n_rows, p.rows), replace=False)).astype(np.int64)
+    p1 = copy.copy(p)
+    p1.h_q, p1.h_kv = p.h_q // p.h_kv, 1
+    d = p.head_dim
+    q = W.round_to_bf16(rng.standard_normal((len(rows), p1.h_q, d), dtype=np.float32) * 0.5)
+    k = W.round_to_bf16(rng.standard_normal((p.rows, 1, d), dtype=np.float32) * 0.5)
+    v = W.round_to_bf16(rng.standard_normal((p.rows, 1, d), dtype=np.float32) * 0.5)
+    go = W.round_to_bf16(rng.standard_normal((len(rows), p1.h_q, d), dtype=np.float32) * 0.1)
+    return p1, rows, q, k, v, go
+
+
+def sample_pairs(oracle, p1, rows):
+    cu = p1.cu_seqlens.astype(np.int64)
+    n = p1.n_main
+    anchors = p1.anchor_idx.astype(np.int64)
+    offs = p1.branch_offsets.astype(np.int64)
+    loc = W.branch_local_counts(p1) if p1.n_branch and p1.n_branch <= 1 << 16 else None
+    total = 0
+    for r in rows:
+        if r < n:
+            s = np.searchsorted(cu, r, side="right") - 1
+            total += r - cu[s] + 1
+        else:
+            tkn = r - n
+            b = np.searchsorted(offs, tkn, side="right") - 1
+            a = anchors[b]
+            s = np.searchsorted(cu, a, side="right") - 1
+            total += a - cu[s] + 1
+            if loc is not None:
+                total += loc[tkn]
+            elif p1.kind == W.CHAIN:
+                total += tkn - offs[b] + 1
+            else:
+                total += offs[b + 1] - offs[b]
+    return int(total)
+
+
+def time_oracle(p, n_rows, backward=True):
+    from oracle import oracle
+    oracle.build()
+    p1, rows, q, k, v, go = oracle_sample(p, n_rows)
+    pairs = sample_pairs(oracle, p1, rows)
+    t0 = time.perf_counter()
+    if backward:
+        oracle.backward(p1, q, k, v, go, rows=rows)       # runs the forward inside
+    else:
+        oracle.forward(p1, q, k, v, rows=rows)
+    dt = time.perf_counter() - t0
+    fl = pairs * 4 * p.head_dim * p1.h_q * (3.5 if backward else 1.0)
+    return fl / dt / 1e12, dt, len(rows), pairs, p1.h_q
+
+
+def cpu_baseline(p, seconds_target=15.0, backward=True):
+    cores = len(os.sched_getaffinity(0))
+    # calibrate on a few rows, then size the sample for ~seconds_target
+    _, dt, nr, pairs, _ = time_oracle(p, 4, backward)
+    n_rows = int(max(4, min(p.rows, 4 * seconds_target / max(dt, 1e-3))))
+    val, dt, nr, pairs, hq = time_oracle(p, n_rows, backward)
+    return {"value": float(f"{val:.6g}"), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{nr} uniformly sampled query rows x {hq} query heads of one KV group, "
+                      f"fwd{'+bwd' if backward else ''}, {pairs} visible pairs per head, {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    name = "config5_256k_zigzag" if args.workload == "auto" else args.workload
+    cfg, shrink, cp, backward = WORKLOADS[name]
+    p = W.CONFIGS[cfg](shrink)
+    cores = len(os.sched_getaffinity(0))
+    _, dt, _, _, _ = time_oracle(p, 4, backward)
+    n_rows = int(max(4, min(p.rows, 4 * args.ref_seconds / max(dt, 1e-3))))
+    for _ in range(args.warmup):
+        time_oracle(p, 4, backward)
+    vals, secs = [], []
+    for _ in range(args.steps):
+        val, dt, nr, pairs, hq = time_oracle(p, n_rows, backward)
+        vals.append(val)
+        secs.append(dt)
+    value = sum(vals) / len(vals)
+    sample = (f"{nr} uniformly sampled query rows x {hq} query heads of one KV group per step, "
+              f"fwd{'+bwd' if backward else ''}, {pairs} visible pairs per head")
+    line = {"impl": "reference", "metric": METRIC, "value": float(f"{value:.6g}"), "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(1e3 * sum(secs) / len(secs), 1), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, "n_main": p.n_main, "rows": p.rows, "h_q": p.h_q, "h_kv": p.h_kv,
+                       "head_dim": p.head_dim, "mask": W.KIND_NAMES[p.kind]},
+            "cpu_baseline": {"value": float(f"{value:.6g}"), "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": float(f"{value:.6g}"), "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="auto", choices=["auto", *WORKLOADS])
+    ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-seconds", type=float, default=8.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,183 @@
+/*
+ * branch_attn.h -- C ABI of the B200 (sm_100a) draft-branch-attention library.
+ *
+ * The operation (paper Section 3.2, "Branch Attention under Context
+ * Parallelism"): over a packed batch of variable-length main sequences, every
+ * main query attends causally inside its own sequence, and every branch query
+ * attends to two key sets -- the causal prefix of its main sequence up to and
+ * including its anchor, and the keys of its own branch under a branch-local
+ * mask (EAGLE-3 chain, DFlash block, or a tree given by parent indices).
+ * Partial results over disjoint key sets are combined with Eq. (lse-merge);
+ * the backward pass accumulates gradients over key chunks.
+ *
+ * Conventions
+ *   - Every pointer marked "device" is CUDA device memory owned by the caller;
+ *     the library allocates no device memory.  `stream` is a cudaStream_t
+ *     passed as void* (NULL = the legacy default stream).  Data calls only
+ *     enqueue work on that stream and return; ba_plan_create synchronises the
+ *     stream once to read back its validation result.
+ *   - Tensors are contiguous, row-major, innermost dimension head_dim:
+ *       q_main  [N, h_q, D]      q_branch [M, h_q, D]
+ *       k, v    [N + M, h_kv, D] main rows first, then branch tokens
+ *       O, dO   [N + M, h_q, D]  LSE [N + M, h_q] (fp32, natural log)
+ *     Branch tokens are stored branch-major in anchor order.  Query head h uses
+ *     KV head h / (h_q / h_kv).
+ *   - Element type of q/k/v/O/dO is ba_problem_t.dtype.  Supported: BA_FP32 and
+ *     BA_BF16 with head_dim 64 or 128; a branch holds at most 64 tokens.
+ *   - Every function returns BA_OK (0) or a negative ba_status; nothing throws.
+ */
+#ifndef BRANCH_ATTN_H_
+#define BRANCH_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum ba_status {
+    BA_OK = 0,
+    BA_EINVAL = -1,        /* bad argument (NULL pointer, negative size, bad range) */
+    BA_EUNSUPPORTED = -2,  /* dtype / head_dim / branch length not supported */
+    BA_EWORKSPACE = -3,    /* plan memory or workspace too small / misaligned */
+    BA_EMETA = -4,         /* device-side validation of the metadata failed */
+    BA_ECUDA = -5,         /* a CUDA runtime call failed; see ba_last_cuda_error */
+    BA_ETIMEOUT = -6       /* a bounded device-side wait expired */
+} ba_status;
+
+enum { BA_BF16 = 0, BA_FP32 = 1 };
+enum { BA_MASK_CHAIN = 0, BA_MASK_BLOCK = 1, BA_MASK_TREE = 2 };
+enum { BA_PART_MAIN = 1, BA_PART_BRANCH = 2 };
+enum { BA_OP_FWD = 0, BA_OP_BWD = 1 };
+
+/* Which kernels a plan uses: the tensor-core (tcgen05) path where the shape
+ * allows it (bf16, head_dim 128), or the plain-FMA path (any supported shape;
+ * the only path for fp32). */
+enum { BA_IMPL_AUTO = 0, BA_IMPL_SIMT = 1, BA_IMPL_TC = 2 };
+
+typedef struct ba_problem {
+    int64_t n_main;                /* N: packed main tokens */
+    int64_t n_branch;              /* M: branch tokens (sum of branch lengths) */
+    int32_t num_seqs;              /* B */
+    int32_t num_branches;          /* A */
+    int32_t h_q, h_kv, head_dim;
+    int32_t dtype;                 /* BA_BF16 / BA_FP32 */
+    float softmax_scale;           /* 0 => 1/sqrt(head_dim) */
+    int32_t mask_kind;             /* BA_MASK_* */
+    int32_t uniform_len;           /* > 0: every branch has this many tokens and
+                                      branch_offsets may be NULL */
+    int32_t impl;                  /* BA_IMPL_* */
+    const int32_t *cu_seqlens;     /* device [B+1], cu[0] = 0, cu[B] = N, non-decreasing */
+    const int32_t *anchor_idx;     /* device [A], global packed index in [0, N), non-decreasing */
+    const int32_t *branch_offsets; /* device [A+1] token offsets (0 .. M), or NULL with uniform_len */
+    const int32_t *parent;         /* device [M], BA_MASK_TREE only: branch-local parent index,
+                                      -1 = root, parent[i] < i */
+} ba_problem_t;
+
+typedef struct ba_plan ba_plan_t;  /* opaque; host object owned by the library */
+
+const char *ba_status_string(int status);
+/* cudaError_t of the most recent failed CUDA call on this thread (0 if none). */
+int ba_last_cuda_error(void);
+
+/*
+ * Metadata builder ("varlen packing and anchor / branch-mask metadata").
+ * ba_plan_bytes: device bytes the plan needs for the given sizes (only the
+ *   integer fields of *p are read).
+ * ba_plan_create: validates *p, derives per-row key bounds, per-token branch
+ *   start and 64-bit branch masks, per-key query ranges (for dK/dV) into
+ *   `plan_mem` (device, 256-byte aligned, >= ba_plan_bytes), synchronises
+ *   `stream`, and returns a host handle in *out.  The metadata arrays in *p
+ *   must stay alive only until this call returns; plan_mem until
+ *   ba_plan_destroy.  Bad metadata (unsorted anchors, anchor out of range,
+ *   parent[i] >= i, branch longer than 64, offsets not ending at M) gives
+ *   BA_EMETA and no plan; no data kernel ever sees unvalidated metadata.
+ * ba_plan_destroy: frees the host handle (not plan_mem).
+ */
+size_t ba_plan_bytes(const ba_problem_t *p);
+int ba_plan_create(const ba_problem_t *p, void *plan_mem, size_t plan_bytes, void *stream,
+                   ba_plan_t **out);
+int ba_plan_destroy(ba_plan_t *plan);
+
+/* Scratch bytes (device, 256-byte aligned) that `op` needs; may be 0. */
+size_t ba_workspace_bytes(const ba_plan_t *plan, int op);
+
+/* Exact number of (query row, visible key) pairs per query head of the whole
+ * problem, as counted by the metadata builder (host value). */
+int64_t ba_plan_pairs(const ba_plan_t *plan);
+
+/* Which kernels the plan resolved to: BA_IMPL_SIMT or BA_IMPL_TC. */
+int ba_plan_impl(const ba_plan_t *plan);
+
+/*
+ * Forward, both key sets fused in one online-softmax pass (Section 3.2: the
+ * causal main-sequence component and the branch-local component; Eq.
+ * (lse-merge) applied tile by tile).
+ *   q_main may be NULL: only branch queries are computed (rows [N, N+M) of the
+ *   outputs are written).  O has the input dtype, LSE is fp32.
+ */
+int branch_attn_fwd(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                    const void *k, const void *v, void *O, float *LSE,
+                    void *workspace, size_t ws_bytes, void *stream);
+
+/*
+ * Partial forward over an explicit key set: one ring step of the packed
+ * zigzag-ring layout of Section 3.2, emulated on one GPU.
+ *   queries: main rows [qm_begin, qm_end) and the tokens of branches
+ *            [br_begin, br_end); either range may be empty.
+ *   keys:    main keys [kv_begin, kv_end) if parts & BA_PART_MAIN (still limited
+ *            to each query's causal prefix), own-branch keys if parts &
+ *            BA_PART_BRANCH.
+ *   outputs: compact, fp32: O_part [(qm_end-qm_begin) + T, h_q, D] and
+ *            LSE_part [.., h_q], main range first, then the T branch tokens.  A
+ *            query that sees no key in the set gets LSE = -inf and O = 0.
+ */
+int branch_attn_fwd_partial(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                            const void *k, const void *v,
+                            int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                            int64_t kv_begin, int64_t kv_end, int parts,
+                            float *O_part, float *LSE_part,
+                            void *workspace, size_t ws_bytes, void *stream);
+
+/*
+ * Eq. (lse-merge):  l = log(e^la + e^lb),  O = e^(la-l) Oa + e^(lb-l) Ob,
+ * evaluated in max-subtracted form; la = lb = -inf gives l = -inf, O = 0.
+ *   rows_heads = number of (row, head) pairs; O_a/O_b fp32 [rows_heads, d],
+ *   LSE_* fp32 [rows_heads].  O_out has out_dtype (BA_FP32 / BA_BF16) and may
+ *   alias O_a when out_dtype is BA_FP32; LSE_out may alias LSE_a or be NULL.
+ */
+int lse_merge(int64_t rows_heads, int d, const float *O_a, const float *LSE_a,
+              const float *O_b, const float *LSE_b, void *O_out, int out_dtype,
+              float *LSE_out, void *stream);
+
+/*
+ * Backward (Section 3.2: "replays the same K/V ring and accumulates gradients
+ * locally").  Loss = sum_r <dO_r, O_r>.  O and LSE are the COMPLETE forward
+ * results (after all merges), global layout; the query / key ranges and
+ * `parts` select which (query, key) terms this call adds, exactly as in
+ * branch_attn_fwd_partial.  Full ranges with accumulate = 0 give the whole
+ * gradient in one call.
+ *   accumulate = 0: dQ_main [N,h_q,D], dQ_branch [M,h_q,D], dK, dV [N+M,h_kv,D]
+ *     have the input dtype; rows of the selected query range (dQ) and of the
+ *     selected key set (dK, dV) are overwritten, all other rows untouched.
+ *   accumulate = 1: the four outputs are fp32 and the terms are added to them
+ *     (the caller zeroes them first and converts with ba_finalize_grads).
+ *   q_main NULL: branch queries only (dQ_main untouched, may be NULL).
+ *   workspace: ba_workspace_bytes(plan, BA_OP_BWD).
+ */
+int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                    const void *k, const void *v, const void *O, const float *LSE,
+                    const void *dO,
+                    int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                    int64_t kv_begin, int64_t kv_end, int parts, int accumulate,
+                    void *dQ_main, void *dQ_branch, void *dK, void *dV,
+                    void *workspace, size_t ws_bytes, void *stream);
+
+/* fp32 accumulators -> dst_dtype (round to nearest even), `count` elements. */
+int ba_finalize_grads(const float *src, void *dst, int64_t count, int dst_dtype, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BRANCH_ATTN_H_ */

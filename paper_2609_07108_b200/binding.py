@@ -1,0 +1,259 @@
+"""Thin ctypes binding of the C-ABI library (`include/branch_attn.h`).
+
+Argument marshalling only: torch provides device memory and streams, every
+step of the computation runs in the library's CUDA kernels.  Importing this
+module fails loudly if the compiled library is missing -- there is no CPU or
+framework fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+BA_BF16, BA_FP32 = 0, 1
+PART_MAIN, PART_BRANCH, PART_ALL = 1, 2, 3
+OP_FWD, OP_BWD = 0, 1
+IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
+
+_DT = {"bf16": (BA_BF16, torch.bfloat16), "fp32": (BA_FP32, torch.float32)}
+
+
+class BranchAttnError(RuntimeError):
+    def __init__(self, code, what):
+        self.code = code
+        super().__init__(f"{what}: {_lib().ba_status_string(code).decode()} (status {code}, "
+                         f"cuda error {_lib().ba_last_cuda_error()})")
+
+
+class _Problem(C.Structure):
+    _fields_ = [
+        ("n_main", C.c_int64), ("n_branch", C.c_int64),
+        ("num_seqs", C.c_int32), ("num_branches", C.c_int32),
+        ("h_q", C.c_int32), ("h_kv", C.c_int32), ("head_dim", C.c_int32),
+        ("dtype", C.c_int32), ("softmax_scale", C.c_float),
+        ("mask_kind", C.c_int32), ("uniform_len", C.c_int32), ("impl", C.c_int32),
+        ("cu_seqlens", C.c_void_p), ("anchor_idx", C.c_void_p),
+        ("branch_offsets", C.c_void_p), ("parent", C.c_void_p),
+    ]
+
+
+_LIB = None
+EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
+           "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "branch_attn_fwd",
+           "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd", "ba_finalize_grads")
+
+
+def _lib():
+    global _LIB
+    if _LIB is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build it with "
+                              "`python -m paper_2609_07108_b200.build` (needs nvcc); "
+                              "there is no fallback path")
+        lib = C.CDLL(path)
+        lib.ba_status_string.restype = C.c_char_p
+        lib.ba_status_string.argtypes = [C.c_int]
+        lib.ba_last_cuda_error.restype = C.c_int
+        lib.ba_plan_bytes.restype = C.c_size_t
+        lib.ba_plan_bytes.argtypes = [C.POINTER(_Problem)]
+        lib.ba_plan_create.restype = C.c_int
+        lib.ba_plan_create.argtypes = [C.POINTER(_Problem), C.c_void_p, C.c_size_t, C.c_void_p,
+                                       C.POINTER(C.c_void_p)]
+        lib.ba_plan_destroy.restype = C.c_int
+        lib.ba_plan_destroy.argtypes = [C.c_void_p]
+        lib.ba_workspace_bytes.restype = C.c_size_t
+        lib.ba_workspace_bytes.argtypes = [C.c_void_p, C.c_int]
+        lib.ba_plan_pairs.restype = C.c_int64
+        lib.ba_plan_pairs.argtypes = [C.c_void_p]
+        lib.ba_plan_impl.restype = C.c_int
+        lib.ba_plan_impl.argtypes = [C.c_void_p]
+        vp, i64 = C.c_void_p, C.c_int64
+        lib.branch_attn_fwd.restype = C.c_int
+        lib.branch_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        lib.branch_attn_fwd_partial.restype = C.c_int
+        lib.branch_attn_fwd_partial.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64,
+                                                C.c_int, vp, vp, vp, C.c_size_t, vp]
+        lib.lse_merge.restype = C.c_int
+        lib.lse_merge.argtypes = [i64, C.c_int, vp, vp, vp, vp, vp, C.c_int, vp, vp]
+        lib.branch_attn_bwd.restype = C.c_int
+        lib.branch_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64,
+                                        C.c_int, C.c_int, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        lib.ba_finalize_grads.restype = C.c_int
+        lib.ba_finalize_grads.argtypes = [vp, vp, i64, C.c_int, vp]
+        _LIB = lib
+    return _LIB
+
+
+def _p(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise BranchAttnError(rc, what)
+
+
+def _dev_i32(a, device):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+
+
+class Plan:
+    """ba_plan_create: metadata builder for one packed batch.
+
+    `problem` is a `workloads.Problem` (host numpy metadata); the arrays are
+    copied to the device, validated and expanded there.
+    """
+
+    def __init__(self, problem, device="cuda", impl=IMPL_AUTO):
+        lib = _lib()
+        self.problem = problem
+        self.device = torch.device(device)
+        self.dtype_code, self.torch_dtype = _DT[problem.dtype]
+        offs = np.asarray(problem.branch_offsets, dtype=np.int64)
+        lens = np.diff(offs)
+        uniform = int(lens[0]) if len(lens) and lens[0] > 0 and (lens == lens[0]).all() else 0
+        self._cu = _dev_i32(problem.cu_seqlens, self.device)
+        self._anchor = _dev_i32(problem.anchor_idx, self.device)
+        self._offs = _dev_i32(offs, self.device)
+        self._parent = _dev_i32(problem.parent, self.device) if problem.parent is not None else None
+        self.c = _Problem(problem.n_main, problem.n_branch, problem.num_seqs, problem.num_branches,
+                          problem.h_q, problem.h_kv, problem.head_dim, self.dtype_code,
+                          float(problem.scale), int(problem.kind), uniform, impl,
+                          self._cu.data_ptr(), self._anchor.data_ptr() if len(self._anchor) else None,
+                          self._offs.data_ptr(),
+                          self._parent.data_ptr() if self._parent is not None and len(self._parent) else None)
+        nbytes = lib.ba_plan_bytes(C.byref(self.c))
+        if nbytes == 0:
+            raise BranchAttnError(-2, "ba_plan_bytes")
+        self._mem = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        handle = C.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = lib.ba_plan_create(C.byref(self.c), _p(self._mem), nbytes, _stream(), C.byref(handle))
+        _check(rc, "ba_plan_create")
+        self.handle = handle
+        self.pairs = int(lib.ba_plan_pairs(handle))
+        self.impl = int(lib.ba_plan_impl(handle))
+        self._ws = {}
+
+    def workspace(self, op):
+        if op not in self._ws:
+            n = _lib().ba_workspace_bytes(self.handle, op)
+            self._ws[op] = torch.empty(max(n, 256), dtype=torch.uint8, device=self.device)
+        return self._ws[op]
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib().ba_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # sizes
+    @property
+    def n(self):
+        return self.problem.n_main
+
+    @property
+    def m(self):
+        return self.problem.n_branch
+
+    def token_range(self, br_begin, br_end):
+        o = self.problem.branch_offsets
+        return int(o[br_begin]), int(o[br_end])
+
+
+def branch_attn_fwd(plan, q_main, q_branch, k, v, out=None, lse=None):
+    """(O [N+M, h_q, D] input dtype, LSE [N+M, h_q] fp32); q_main may be None."""
+    p = plan.problem
+    if out is None:
+        out = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=plan.device)
+    if lse is None:
+        lse = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=plan.device)
+    ws = plan.workspace(OP_FWD)
+    rc = _lib().branch_attn_fwd(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(out), _p(lse),
+                                _p(ws), ws.numel(), _stream())
+    _check(rc, "branch_attn_fwd")
+    return out, lse
+
+
+def branch_attn_fwd_partial(plan, q_main, q_branch, k, v, qm_range, br_range, kv_range, parts,
+                            out=None, lse=None):
+    """Compact fp32 (O_part, LSE_part) of the selected queries over the selected key set."""
+    p = plan.problem
+    t0, t1 = plan.token_range(*br_range)
+    rows = (qm_range[1] - qm_range[0]) + (t1 - t0)
+    if out is None:
+        out = torch.empty((rows, p.h_q, p.head_dim), dtype=torch.float32, device=plan.device)
+    if lse is None:
+        lse = torch.empty((rows, p.h_q), dtype=torch.float32, device=plan.device)
+    ws = plan.workspace(OP_FWD)
+    rc = _lib().branch_attn_fwd_partial(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v),
+                                        qm_range[0], qm_range[1], br_range[0], br_range[1],
+                                        kv_range[0], kv_range[1], parts, _p(out), _p(lse),
+                                        _p(ws), ws.numel(), _stream())
+    _check(rc, "branch_attn_fwd_partial")
+    return out, lse
+
+
+def lse_merge(o_a, lse_a, o_b, lse_b, out=None, lse_out=None, out_dtype=torch.float32):
+    """Eq. (lse-merge); `out` may be `o_a` (fp32, in place)."""
+    d = o_a.shape[-1]
+    items = lse_a.numel()
+    if out is None:
+        out = torch.empty(o_a.shape, dtype=out_dtype, device=o_a.device)
+    if lse_out is None:
+        lse_out = torch.empty_like(lse_a)
+    code = BA_BF16 if out.dtype == torch.bfloat16 else BA_FP32
+    rc = _lib().lse_merge(items, d, _p(o_a), _p(lse_a), _p(o_b), _p(lse_b), _p(out), code,
+                          _p(lse_out), _stream())
+    _check(rc, "lse_merge")
+    return out, lse_out
+
+
+def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br_range=None,
+                    kv_range=None, parts=PART_ALL, accumulate=False, grads=None):
+    """(dQ_main, dQ_branch, dK, dV).  With `accumulate`, `grads` must hold four
+    zero-initialised fp32 tensors which receive the selected terms."""
+    p = plan.problem
+    qm_range = (0, p.n_main) if qm_range is None else qm_range
+    br_range = (0, p.num_branches) if br_range is None else br_range
+    kv_range = (0, p.n_main) if kv_range is None else kv_range
+    if grads is None:
+        dt = torch.float32 if accumulate else plan.torch_dtype
+        mk = torch.zeros if accumulate else torch.empty
+        grads = (mk((p.n_main, p.h_q, p.head_dim), dtype=dt, device=plan.device)
+                 if q_main is not None else None,
+                 mk((p.n_branch, p.h_q, p.head_dim), dtype=dt, device=plan.device),
+                 mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device),
+                 mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device))
+    ws = plan.workspace(OP_BWD)
+    rc = _lib().branch_attn_bwd(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(o), _p(lse),
+                                _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1],
+                                kv_range[0], kv_range[1], parts, 1 if accumulate else 0,
+                                _p(grads[0]), _p(grads[1]), _p(grads[2]), _p(grads[3]),
+                                _p(ws), ws.numel(), _stream())
+    _check(rc, "branch_attn_bwd")
+    return grads
+
+
+def ba_finalize_grads(src, dst=None, dtype=torch.bfloat16):
+    if dst is None:
+        dst = torch.empty(src.shape, dtype=dtype, device=src.device)
+    code = BA_BF16 if dst.dtype == torch.bfloat16 else BA_FP32
+    rc = _lib().ba_finalize_grads(_p(src), _p(dst), src.numel(), code, _stream())
+    _check(rc, "ba_finalize_grads")
+    return dst

@@ -1,0 +1,119 @@
+// C-ABI entry points: argument checks and dispatch to the plain-FMA or the
+// tensor-core kernels.  No device memory is allocated here; every call only
+// enqueues kernels on the caller's stream.
+#include "ba_common.cuh"
+
+namespace {
+
+inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// Branch index range -> branch token range.
+int token_range(const ba_plan *pl, int64_t br_begin, int64_t br_end, int64_t *t0, int64_t *t1) {
+    const int64_t a = pl->prob.num_branches;
+    if (br_begin < 0 || br_end < br_begin || br_end > a) return BA_EINVAL;
+    if (pl->prob.uniform_len > 0) {
+        *t0 = br_begin * pl->prob.uniform_len;
+        *t1 = br_end * pl->prob.uniform_len;
+    } else if (a > 0) {
+        *t0 = pl->host_offsets[br_begin];
+        *t1 = pl->host_offsets[br_end];
+    } else {
+        *t0 = *t1 = 0;
+    }
+    return BA_OK;
+}
+
+int make_range(const ba_plan *pl, int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+               int64_t kv_begin, int64_t kv_end, int parts, BaRange *r) {
+    const int64_t n = pl->prob.n_main;
+    if (qm_begin < 0 || qm_end < qm_begin || qm_end > n) return BA_EINVAL;
+    if (kv_begin < 0 || kv_end < kv_begin || kv_end > n) return BA_EINVAL;
+    if (parts < 0 || parts > (BA_PART_MAIN | BA_PART_BRANCH)) return BA_EINVAL;
+    r->qm_begin = qm_begin; r->qm_end = qm_end;
+    r->kv_begin = kv_begin; r->kv_end = kv_end;
+    r->parts = parts;
+    return token_range(pl, br_begin, br_end, &r->tok_begin, &r->tok_end);
+}
+
+}  // namespace
+
+extern "C" size_t ba_workspace_bytes(const ba_plan_t *plan, int op) {
+    if (!plan) return 0;
+    if (op == BA_OP_BWD)  // delta = rowsum(dO * O), fp32 [N + M, h_q]
+        return align256((size_t)(plan->prob.n_main + plan->prob.n_branch) * plan->prob.h_q * sizeof(float));
+    return 0;
+}
+
+static int fwd_common(const ba_plan_t *plan, const BaRange &r, const void *q_main, const void *q_branch,
+                      const void *k, const void *v, void *o, float *lse, bool partial, void *stream) {
+    const bool has_main_q = q_main != nullptr && r.qm_end > r.qm_begin;
+    const bool has_branch_q = r.tok_end > r.tok_begin;
+    if (!has_main_q && !has_branch_q) return BA_OK;
+    if (!k || !v || !o || !lse) return BA_EINVAL;
+    if (has_branch_q && !q_branch) return BA_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (plan->impl == BA_IMPL_TC) return ba_tc_fwd(plan, r, q_main, q_branch, k, v, o, lse, partial, st);
+    return ba_simt_fwd(plan, r, q_main, q_branch, k, v, o, lse, partial, st);
+}
+
+extern "C" int branch_attn_fwd(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                               const void *k, const void *v, void *O, float *LSE, void *workspace,
+                               size_t ws_bytes, void *stream) {
+    (void)workspace; (void)ws_bytes;
+    if (!plan) return BA_EINVAL;
+    BaRange r;
+    int rc = make_range(plan, 0, plan->prob.n_main, 0, plan->prob.num_branches, 0, plan->prob.n_main,
+                        BA_PART_MAIN | BA_PART_BRANCH, &r);
+    if (rc != BA_OK) return rc;
+    return fwd_common(plan, r, q_main, q_branch, k, v, O, LSE, false, stream);
+}
+
+extern "C" int branch_attn_fwd_partial(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                                       const void *k, const void *v, int64_t qm_begin, int64_t qm_end,
+                                       int64_t br_begin, int64_t br_end, int64_t kv_begin,
+                                       int64_t kv_end, int parts, float *O_part, float *LSE_part,
+                                       void *workspace, size_t ws_bytes, void *stream) {
+    (void)workspace; (void)ws_bytes;
+    if (!plan) return BA_EINVAL;
+    BaRange r;
+    int rc = make_range(plan, qm_begin, qm_end, br_begin, br_end, kv_begin, kv_end, parts, &r);
+    if (rc != BA_OK) return rc;
+    if (!q_main && qm_end > qm_begin) return BA_EINVAL;
+    return fwd_common(plan, r, q_main, q_branch, k, v, O_part, LSE_part, true, stream);
+}
+
+extern "C" int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                               const void *k, const void *v, const void *O, const float *LSE,
+                               const void *dO, int64_t qm_begin, int64_t qm_end, int64_t br_begin,
+                               int64_t br_end, int64_t kv_begin, int64_t kv_end, int parts,
+                               int accumulate, void *dQ_main, void *dQ_branch, void *dK, void *dV,
+                               void *workspace, size_t ws_bytes, void *stream) {
+    if (!plan) return BA_EINVAL;
+    BaRange r;
+    int rc = make_range(plan, qm_begin, qm_end, br_begin, br_end, kv_begin, kv_end, parts, &r);
+    if (rc != BA_OK) return rc;
+    if (!q_main) r.qm_end = r.qm_begin;  // branch queries only
+    const bool has_main_q = r.qm_end > r.qm_begin;
+    const bool has_branch_q = r.tok_end > r.tok_begin;
+    if (!has_main_q && !has_branch_q) return BA_OK;
+    if (!k || !v || !O || !LSE || !dO || !dK || !dV) return BA_EINVAL;
+    if (has_main_q && !dQ_main) return BA_EINVAL;
+    if (has_branch_q && (!q_branch || !dQ_branch)) return BA_EINVAL;
+    if (accumulate != 0 && accumulate != 1) return BA_EINVAL;
+    const size_t need = ba_workspace_bytes(plan, BA_OP_BWD);
+    if (!workspace || ws_bytes < need || ((uintptr_t)workspace & 255)) return BA_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    float *delta = (float *)workspace;
+    const int64_t n = plan->prob.n_main;
+    const int hq = plan->prob.h_q, d = plan->prob.head_dim, dt = plan->prob.dtype;
+    if (has_main_q && (rc = ba_delta(O, dO, delta, r.qm_begin, r.qm_end, hq, d, dt, st)) != BA_OK) return rc;
+    if (has_branch_q &&
+        (rc = ba_delta(O, dO, delta, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
+        return rc;
+    const void *qm = has_main_q ? q_main : nullptr;
+    if (plan->impl == BA_IMPL_TC)
+        return ba_tc_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK,
+                         dV, st);
+    return ba_simt_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK, dV,
+                       st);
+}

@@ -1,0 +1,477 @@
+// Plain-FMA (CUDA-core) branch attention: forward, dQ and dK/dV kernels.
+//
+// This is the fp32 path (tensor cores cannot meet a 1e-4 absolute bound on
+// N(0,1) inputs in a single tf32 pass) and the fallback for every supported
+// shape.  Same metadata and same semantics as the tensor-core path: both key
+// sets of a branch query (causal main prefix, own-branch keys; paper Section
+// 3.2) go through ONE online-softmax pass, i.e. Eq. (lse-merge) applied key
+// by key.
+//
+// Work split: TPR = D/32 threads share one row (query row, or key row in the
+// dK/dV kernel); each thread keeps 32 of the row's D elements in registers as
+// eight float4 chunks interleaved across the TPR threads, so that shared-memory
+// reads of the opposite operand are 16-byte, conflict-free broadcasts.
+#include <limits.h>
+#include <string.h>
+
+#include "ba_common.cuh"
+
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kKeyTile = 32;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct SimtArgs {
+    BaMeta meta;
+    BaRange r;
+    const void *q_main, *q_branch, *k, *v, *d_o;
+    const float *lse_in, *delta;
+    void *o;          // forward output
+    float *lse_out;
+    void *dq_main, *dq_branch, *dk, *dv;
+    int h_q, h_kv;
+    float scale, scale_log2;
+    int partial_out;  // forward: compact fp32 outputs
+    int accumulate;   // backward: fp32 += outputs
+    int64_t main_tiles;
+};
+
+template <typename T> __device__ __forceinline__ float4 load4(const T *p);
+template <> __device__ __forceinline__ float4 load4<float>(const float *p) {
+    return *reinterpret_cast<const float4 *>(p);
+}
+template <> __device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16 *p) {
+    const uint2 raw = *reinterpret_cast<const uint2 *>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+template <typename T> __device__ __forceinline__ void store4(T *p, float4 x);
+template <> __device__ __forceinline__ void store4<float>(float *p, float4 x) {
+    *reinterpret_cast<float4 *>(p) = x;
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 *p, float4 x) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+    uint2 r;
+    r.x = *reinterpret_cast<uint32_t *>(&lo);
+    r.y = *reinterpret_cast<uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = r;
+}
+
+template <int TPR> __device__ __forceinline__ float group_sum(float x) {
+    x += __shfl_xor_sync(0xffffffffu, x, 1);
+    if (TPR == 4) x += __shfl_xor_sync(0xffffffffu, x, 2);
+    return x;
+}
+
+// rows [tile_first, tile_first + count) of `src` ([rows, heads, D]) for `head`
+// -> fp32 shared tile [count][D]; rows beyond `count` are not touched.
+template <typename T, int D>
+__device__ __forceinline__ void load_tile(float *dst, const T *src, int64_t first, int count,
+                                          int heads, int head) {
+    constexpr int CPR = D / 4;  // float4 chunks per row
+    for (int idx = threadIdx.x; idx < count * CPR; idx += kThreads) {
+        const int row = idx / CPR, ch = idx % CPR;
+        const float4 x = load4<T>(src + ((size_t)(first + row) * heads + head) * D + ch * 4);
+        *reinterpret_cast<float4 *>(dst + row * D + ch * 4) = x;
+    }
+}
+
+// ------------------------------------------------------------------ forward / dQ
+// MODE 0: forward (O, LSE);  MODE 1: dQ.
+template <typename T, int D, int MODE>
+__global__ void __launch_bounds__(kThreads) simt_row_kernel(const SimtArgs a) {
+    constexpr int TPR = D / 32;
+    constexpr int RB = kThreads / TPR;
+    __shared__ __align__(16) float k_s[kKeyTile * D];
+    __shared__ __align__(16) float v_s[kKeyTile * D];
+    __shared__ int s_lo, s_hi, s_bs, s_be;
+
+    const int tid = threadIdx.x, c = tid % TPR, rl = tid / TPR;
+    const int h = blockIdx.y, g = h / (a.h_q / a.h_kv);
+    const bool is_main = (int64_t)blockIdx.x < a.main_tiles;
+    const int64_t n = a.meta.n_main;
+    int64_t row;  // index into the main rows, or into the branch tokens
+    bool valid;
+    if (is_main) {
+        row = a.r.qm_begin + (int64_t)blockIdx.x * RB + rl;
+        valid = row < a.r.qm_end;
+    } else {
+        row = a.r.tok_begin + ((int64_t)blockIdx.x - a.main_tiles) * RB + rl;
+        valid = row < a.r.tok_end;
+    }
+    const int64_t grow = is_main ? row : n + row;  // global row
+
+    if (tid == 0) { s_lo = INT_MAX; s_hi = -1; s_bs = INT_MAX; s_be = -1; }
+    __syncthreads();
+    int lo = 0, hi = -1, bstart = 0;
+    uint64_t mask = 0;
+    if (valid) {
+        lo = max(a.meta.row_lo[grow], (int)a.r.kv_begin);
+        hi = min(a.meta.row_hi[grow], (int)a.r.kv_end - 1);
+        if (!(a.r.parts & BA_PART_MAIN)) { lo = 0; hi = -1; }
+        if (!is_main && (a.r.parts & BA_PART_BRANCH)) {
+            bstart = a.meta.br_start[row];
+            mask = a.meta.br_mask[row];
+            if (c == 0) { atomicMin(&s_bs, bstart); atomicMax(&s_be, a.meta.br_end[row]); }
+        }
+        if (c == 0 && hi >= lo) { atomicMin(&s_lo, lo); atomicMax(&s_hi, hi); }
+    }
+
+    float q[32], acc[32];  // acc: O accumulator (forward) or dQ accumulator
+    float go[MODE == 1 ? 32 : 1];
+    float m = -INFINITY, l = 0.f, lse2 = 0.f, dlt = 0.f;
+#pragma unroll
+    for (int e = 0; e < 32; ++e) { q[e] = 0.f; acc[e] = 0.f; }
+    if (valid) {
+        const T *qp = is_main ? (const T *)a.q_main + ((size_t)row * a.h_q + h) * D
+                              : (const T *)a.q_branch + ((size_t)row * a.h_q + h) * D;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float4 x = load4<T>(qp + (e * TPR + c) * 4);
+            q[4 * e] = x.x; q[4 * e + 1] = x.y; q[4 * e + 2] = x.z; q[4 * e + 3] = x.w;
+        }
+        if (MODE == 1) {
+            const T *gp = (const T *)a.d_o + ((size_t)grow * a.h_q + h) * D;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float4 x = load4<T>(gp + (e * TPR + c) * 4);
+                go[4 * e] = x.x; go[4 * e + 1] = x.y; go[4 * e + 2] = x.z; go[4 * e + 3] = x.w;
+            }
+            lse2 = a.lse_in[grow * a.h_q + h] * kLog2e;
+            dlt = a.delta[grow * a.h_q + h];
+        }
+    }
+    __syncthreads();
+
+    // phase 0: main keys [s_lo, s_hi];  phase 1: own-branch keys [s_bs, s_be)
+    for (int phase = 0; phase < 2; ++phase) {
+        int64_t key0, key1;  // global key rows
+        if (phase == 0) { key0 = s_lo; key1 = (int64_t)s_hi + 1; }
+        else { key0 = n + s_bs; key1 = n + s_be; }
+        if (phase == 1 && is_main) break;
+        for (int64_t kt = key0; kt < key1; kt += kKeyTile) {
+            const int cnt = (int)min((int64_t)kKeyTile, key1 - kt);
+            __syncthreads();
+            load_tile<T, D>(k_s, (const T *)a.k, kt, cnt, a.h_kv, g);
+            load_tile<T, D>(v_s, (const T *)a.v, kt, cnt, a.h_kv, g);
+            __syncthreads();
+            for (int j = 0; j < cnt; ++j) {
+                const float4 *kr = reinterpret_cast<const float4 *>(k_s + j * D);
+                const float4 *vr = reinterpret_cast<const float4 *>(v_s + j * D);
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float4 kk = kr[e * TPR + c];
+                    s += q[4 * e] * kk.x + q[4 * e + 1] * kk.y + q[4 * e + 2] * kk.z + q[4 * e + 3] * kk.w;
+                }
+                s = group_sum<TPR>(s);
+                float dp = 0.f;
+                if (MODE == 1) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 vv = vr[e * TPR + c];
+                        dp += go[4 * e] * vv.x + go[4 * e + 1] * vv.y + go[4 * e + 2] * vv.z + go[4 * e + 3] * vv.w;
+                    }
+                    dp = group_sum<TPR>(dp);
+                }
+                bool vis;
+                if (phase == 0) {
+                    const int x = (int)(kt + j);
+                    vis = valid && x >= lo && x <= hi;
+                } else {
+                    const int rel = (int)(kt + j - n) - bstart;
+                    vis = valid && rel >= 0 && rel < 64 && ((mask >> rel) & 1ull);
+                }
+                if (!vis) continue;
+                if (MODE == 0) {
+                    const float s2 = s * a.scale_log2;
+                    if (s2 > m) {
+                        const float alpha = exp2f(m - s2);
+                        l *= alpha;
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) acc[e] *= alpha;
+                        m = s2;
+                    }
+                    const float p = exp2f(s2 - m);
+                    l += p;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 vv = vr[e * TPR + c];
+                        acc[4 * e] += p * vv.x; acc[4 * e + 1] += p * vv.y;
+                        acc[4 * e + 2] += p * vv.z; acc[4 * e + 3] += p * vv.w;
+                    }
+                } else {
+                    const float p = exp2f(s * a.scale_log2 - lse2);
+                    const float ds = p * (dp - dlt);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 kk = kr[e * TPR + c];
+                        acc[4 * e] += ds * kk.x; acc[4 * e + 1] += ds * kk.y;
+                        acc[4 * e + 2] += ds * kk.z; acc[4 * e + 3] += ds * kk.w;
+                    }
+                }
+            }
+        }
+    }
+    if (!valid) return;
+
+    if (MODE == 0) {
+        const float inv = l > 0.f ? 1.0f / l : 0.f;
+        int64_t orow = grow;
+        if (a.partial_out)
+            orow = is_main ? row - a.r.qm_begin : (a.r.qm_end - a.r.qm_begin) + (row - a.r.tok_begin);
+        if (c == 0) a.lse_out[orow * a.h_q + h] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+        const size_t base = ((size_t)orow * a.h_q + h) * D;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float4 x = make_float4(acc[4 * e] * inv, acc[4 * e + 1] * inv, acc[4 * e + 2] * inv,
+                                         acc[4 * e + 3] * inv);
+            if (a.partial_out) store4<float>((float *)a.o + base + (e * TPR + c) * 4, x);
+            else store4<T>((T *)a.o + base + (e * TPR + c) * 4, x);
+        }
+    } else {
+        void *dst = is_main ? a.dq_main : a.dq_branch;
+        const size_t base = ((size_t)row * a.h_q + h) * D;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float4 x = make_float4(acc[4 * e] * a.scale, acc[4 * e + 1] * a.scale,
+                                   acc[4 * e + 2] * a.scale, acc[4 * e + 3] * a.scale);
+            const size_t off = base + (e * TPR + c) * 4;
+            if (a.accumulate) {
+                const float4 old = load4<float>((float *)dst + off);
+                x.x += old.x; x.y += old.y; x.z += old.z; x.w += old.w;
+                store4<float>((float *)dst + off, x);
+            } else {
+                store4<T>((T *)dst + off, x);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ dK / dV
+// One thread group per key row and KV head; loops over the query rows that see
+// the key (all query heads of the KV head), so every output element has one
+// owner and the sums are deterministic.
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads) simt_dkdv_kernel(const SimtArgs a) {
+    constexpr int TPR = D / 32;
+    constexpr int KB = kThreads / TPR;
+    constexpr int QT = 32;
+    __shared__ __align__(16) float q_s[QT * D];
+    __shared__ __align__(16) float g_s[QT * D];
+    __shared__ float lse_s[QT], dlt_s[QT];
+    __shared__ int lo_s[QT], hi_s[QT], bst_s[QT];
+    __shared__ unsigned long long mask_s[QT];
+    __shared__ int s_q1, s_b1, s_b0;
+
+    const int tid = threadIdx.x, c = tid % TPR, kl = tid / TPR;
+    const int g = blockIdx.y, grp = a.h_q / a.h_kv;
+    const int64_t n = a.meta.n_main;
+    const bool main_keys = (int64_t)blockIdx.x < a.main_tiles;
+    int64_t key;  // main key index or branch token index
+    bool valid;
+    if (main_keys) {
+        key = a.r.kv_begin + (int64_t)blockIdx.x * KB + kl;
+        valid = key < a.r.kv_end;
+    } else {
+        key = a.r.tok_begin + ((int64_t)blockIdx.x - a.main_tiles) * KB + kl;
+        valid = key < a.r.tok_end;
+    }
+    const int64_t gkey = main_keys ? key : n + key;
+
+    if (tid == 0) { s_q1 = -1; s_b1 = -1; s_b0 = INT_MAX; }
+    __syncthreads();
+    if (valid && c == 0) {
+        if (main_keys) {
+            atomicMax(&s_q1, a.meta.key_qend[key]);
+            atomicMin(&s_b0, a.meta.key_bq_begin[key]);
+            atomicMax(&s_b1, a.meta.key_bq_end[key]);
+        } else {
+            atomicMin(&s_b0, a.meta.br_start[key]);
+            atomicMax(&s_b1, a.meta.br_end[key]);
+        }
+    }
+    float kk[32], vv[32], dk[32], dv[32];
+#pragma unroll
+    for (int e = 0; e < 32; ++e) { kk[e] = 0.f; vv[e] = 0.f; dk[e] = 0.f; dv[e] = 0.f; }
+    if (valid) {
+        const T *kp = (const T *)a.k + ((size_t)gkey * a.h_kv + g) * D;
+        const T *vp = (const T *)a.v + ((size_t)gkey * a.h_kv + g) * D;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float4 x = load4<T>(kp + (e * TPR + c) * 4), y = load4<T>(vp + (e * TPR + c) * 4);
+            kk[4 * e] = x.x; kk[4 * e + 1] = x.y; kk[4 * e + 2] = x.z; kk[4 * e + 3] = x.w;
+            vv[4 * e] = y.x; vv[4 * e + 1] = y.y; vv[4 * e + 2] = y.z; vv[4 * e + 3] = y.w;
+        }
+    }
+    __syncthreads();
+
+    // query ranges: phase 0 = main query rows, phase 1 = branch tokens
+    const int64_t tile_first_key = main_keys ? a.r.kv_begin + (int64_t)blockIdx.x * KB : 0;
+    for (int phase = 0; phase < 2; ++phase) {
+        int64_t r0, r1;
+        if (phase == 0) {
+            if (!main_keys || a.q_main == nullptr) continue;
+            r0 = max(tile_first_key, a.r.qm_begin);
+            r1 = min((int64_t)s_q1, a.r.qm_end);
+        } else {
+            r0 = max((int64_t)s_b0, a.r.tok_begin);
+            r1 = min((int64_t)s_b1, a.r.tok_end);
+        }
+        for (int hh = 0; hh < grp; ++hh) {
+            const int h = g * grp + hh;
+            for (int64_t rt = r0; rt < r1; rt += QT) {
+                const int cnt = (int)min((int64_t)QT, r1 - rt);
+                const int64_t grow0 = phase == 0 ? rt : n + rt;
+                __syncthreads();
+                load_tile<T, D>(q_s, phase == 0 ? (const T *)a.q_main : (const T *)a.q_branch, rt, cnt,
+                                a.h_q, h);
+                load_tile<T, D>(g_s, (const T *)a.d_o, grow0, cnt, a.h_q, h);
+                if (tid < cnt) {
+                    lse_s[tid] = a.lse_in[(grow0 + tid) * a.h_q + h] * kLog2e;
+                    dlt_s[tid] = a.delta[(grow0 + tid) * a.h_q + h];
+                    lo_s[tid] = a.meta.row_lo[grow0 + tid];
+                    hi_s[tid] = a.meta.row_hi[grow0 + tid];
+                    if (phase == 1) {
+                        bst_s[tid] = a.meta.br_start[rt + tid];
+                        mask_s[tid] = a.meta.br_mask[rt + tid];
+                    }
+                }
+                __syncthreads();
+                for (int j = 0; j < cnt; ++j) {
+                    const float4 *qr = reinterpret_cast<const float4 *>(q_s + j * D);
+                    const float4 *gr = reinterpret_cast<const float4 *>(g_s + j * D);
+                    float s = 0.f, dp = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 x = qr[e * TPR + c], y = gr[e * TPR + c];
+                        s += kk[4 * e] * x.x + kk[4 * e + 1] * x.y + kk[4 * e + 2] * x.z + kk[4 * e + 3] * x.w;
+                        dp += vv[4 * e] * y.x + vv[4 * e + 1] * y.y + vv[4 * e + 2] * y.z + vv[4 * e + 3] * y.w;
+                    }
+                    s = group_sum<TPR>(s);
+                    dp = group_sum<TPR>(dp);
+                    bool vis;
+                    if (main_keys) {
+                        vis = valid && key >= lo_s[j] && key <= hi_s[j];
+                    } else {
+                        const int rel = (int)key - bst_s[j];
+                        vis = valid && rel >= 0 && rel < 64 && ((mask_s[j] >> rel) & 1ull);
+                    }
+                    if (!vis) continue;
+                    const float p = exp2f(s * a.scale_log2 - lse_s[j]);
+                    const float ds = p * (dp - dlt_s[j]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float4 x = qr[e * TPR + c], y = gr[e * TPR + c];
+                        dk[4 * e] += ds * x.x; dk[4 * e + 1] += ds * x.y;
+                        dk[4 * e + 2] += ds * x.z; dk[4 * e + 3] += ds * x.w;
+                        dv[4 * e] += p * y.x; dv[4 * e + 1] += p * y.y;
+                        dv[4 * e + 2] += p * y.z; dv[4 * e + 3] += p * y.w;
+                    }
+                }
+            }
+        }
+    }
+    if (!valid) return;
+    const size_t base = ((size_t)gkey * a.h_kv + g) * D;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        float4 x = make_float4(dk[4 * e] * a.scale, dk[4 * e + 1] * a.scale, dk[4 * e + 2] * a.scale,
+                               dk[4 * e + 3] * a.scale);
+        float4 y = make_float4(dv[4 * e], dv[4 * e + 1], dv[4 * e + 2], dv[4 * e + 3]);
+        const size_t off = base + (e * TPR + c) * 4;
+        if (a.accumulate) {
+            const float4 ox = load4<float>((float *)a.dk + off), oy = load4<float>((float *)a.dv + off);
+            x.x += ox.x; x.y += ox.y; x.z += ox.z; x.w += ox.w;
+            y.x += oy.x; y.y += oy.y; y.z += oy.z; y.w += oy.w;
+            store4<float>((float *)a.dk + off, x);
+            store4<float>((float *)a.dv + off, y);
+        } else {
+            store4<T>((T *)a.dk + off, x);
+            store4<T>((T *)a.dv + off, y);
+        }
+    }
+}
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+SimtArgs base_args(const ba_plan *pl, const BaRange &r) {
+    SimtArgs a;
+    memset(&a, 0, sizeof a);
+    a.meta = pl->meta;
+    a.r = r;
+    a.h_q = pl->prob.h_q;
+    a.h_kv = pl->prob.h_kv;
+    a.scale = pl->scale;
+    a.scale_log2 = pl->scale * kLog2e;
+    return a;
+}
+
+template <typename T, int D>
+int launch_fwd(SimtArgs &a, cudaStream_t st) {
+    constexpr int RB = kThreads / (D / 32);
+    const int64_t mt = a.q_main ? ceil_div(a.r.qm_end - a.r.qm_begin, RB) : 0;
+    const int64_t bt = ceil_div(a.r.tok_end - a.r.tok_begin, RB);
+    a.main_tiles = mt;
+    if (mt + bt == 0) return BA_OK;
+    dim3 grid((unsigned)(mt + bt), (unsigned)a.h_q);
+    simt_row_kernel<T, D, 0><<<grid, kThreads, 0, st>>>(a);
+    return ba_check_launch();
+}
+
+template <typename T, int D>
+int launch_bwd(SimtArgs &a, cudaStream_t st) {
+    constexpr int RB = kThreads / (D / 32);
+    {
+        const int64_t mt = a.q_main ? ceil_div(a.r.qm_end - a.r.qm_begin, RB) : 0;
+        const int64_t bt = ceil_div(a.r.tok_end - a.r.tok_begin, RB);
+        a.main_tiles = mt;
+        if (mt + bt > 0) {
+            dim3 grid((unsigned)(mt + bt), (unsigned)a.h_q);
+            simt_row_kernel<T, D, 1><<<grid, kThreads, 0, st>>>(a);
+            int rc = ba_check_launch();
+            if (rc != BA_OK) return rc;
+        }
+    }
+    {
+        const int64_t mt = (a.r.parts & BA_PART_MAIN) ? ceil_div(a.r.kv_end - a.r.kv_begin, RB) : 0;
+        const int64_t bt = (a.r.parts & BA_PART_BRANCH) ? ceil_div(a.r.tok_end - a.r.tok_begin, RB) : 0;
+        a.main_tiles = mt;
+        if (mt + bt > 0) {
+            dim3 grid((unsigned)(mt + bt), (unsigned)a.h_kv);
+            simt_dkdv_kernel<T, D><<<grid, kThreads, 0, st>>>(a);
+            int rc = ba_check_launch();
+            if (rc != BA_OK) return rc;
+        }
+    }
+    return BA_OK;
+}
+
+}  // namespace
+
+int ba_simt_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
+                const void *k, const void *v, void *o, float *lse, bool partial_out,
+                cudaStream_t st) {
+    SimtArgs a = base_args(pl, r);
+    a.q_main = q_main; a.q_branch = q_branch; a.k = k; a.v = v;
+    a.o = o; a.lse_out = lse; a.partial_out = partial_out ? 1 : 0;
+    const int d = pl->prob.head_dim;
+    if (pl->prob.dtype == BA_FP32) return d == 64 ? launch_fwd<float, 64>(a, st) : launch_fwd<float, 128>(a, st);
+    return d == 64 ? launch_fwd<__nv_bfloat16, 64>(a, st) : launch_fwd<__nv_bfloat16, 128>(a, st);
+}
+
+int ba_simt_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
+                const void *k, const void *v, const float *lse, const float *delta,
+                const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
+                void *dv, cudaStream_t st) {
+    SimtArgs a = base_args(pl, r);
+    a.q_main = q_main; a.q_branch = q_branch; a.k = k; a.v = v; a.d_o = d_o;
+    a.lse_in = lse; a.delta = delta; a.accumulate = accumulate;
+    a.dq_main = dq_main; a.dq_branch = dq_branch; a.dk = dk; a.dv = dv;
+    const int d = pl->prob.head_dim;
+    if (pl->prob.dtype == BA_FP32) return d == 64 ? launch_bwd<float, 64>(a, st) : launch_bwd<float, 128>(a, st);
+    return d == 64 ? launch_bwd<__nv_bfloat16, 64>(a, st) : launch_bwd<__nv_bfloat16, 128>(a, st);
+}

@@ -1,0 +1,225 @@
+"""GPU parity: the CUDA library (through its C ABI / ctypes binding) against
+the fp64 CPU oracle, element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_07108_b200 import workloads as W
+from helpers import (TOL, assert_close, assert_lse_close, f32, oracle_fwd_bwd, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ba():
+    from paper_2609_07108_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+def impls_for(ba, p):
+    out = [ba.IMPL_SIMT]
+    if p.dtype == "bf16" and p.head_dim == 128:
+        out.append(ba.IMPL_TC)
+    return out
+
+
+def check_full(ba, oracle, p, seed=0, std=1.0, impl=None, backward=True, groups=None, q_main=True,
+               mutate=None):
+    """Monolithic forward (+ backward) against the oracle on all rows."""
+    t = W.make_tensors(p, seed=seed, std=std)
+    if mutate:
+        mutate(t)
+    d = to_dev(p, t)
+    plan = ba.Plan(p, impl=impl if impl is not None else ba.IMPL_AUTO)
+    assert plan.pairs == W.useful_pairs(p)
+    n = p.n_main
+    qm = d["q_main"] if q_main else None
+    o, lse = ba.branch_attn_fwd(plan, qm, d["q_branch"], d["k"], d["v"])
+    ref = oracle_fwd_bwd(oracle, p, t, groups=groups, backward=backward)
+    qh, kvh = ref["q_heads"], ref["kv_heads"]
+    tol = TOL[p.dtype]
+    lo = 0 if q_main else n
+    assert_close("O", f32(o)[lo:, qh], ref["o"][lo:], tol)
+    assert_lse_close(f32(lse)[lo:, qh], ref["lse"][lo:])
+    if not backward:
+        return
+    if not q_main:
+        # gradients of the branch rows only: cotangent of main rows is zero
+        t["d_o"][:n] = 0
+        d["d_o"][:n] = 0
+        # the forward left main rows of O/LSE unwritten; the backward must not read them
+        ref = oracle_fwd_bwd(oracle, p, t, groups=groups)
+    dqm, dqb, dk, dv = ba.branch_attn_bwd(plan, qm, d["q_branch"], d["k"], d["v"], o, lse, d["d_o"])
+    if q_main:
+        assert_close("dQ_main", f32(dqm)[:, qh], ref["dq"][:n], tol)
+    assert_close("dQ_branch", f32(dqb)[:, qh], ref["dq"][n:], tol)
+    assert_close("dK", f32(dk)[:, kvh], ref["dk"], tol)
+    assert_close("dV", f32(dv)[:, kvh], ref["dv"], tol)
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ metadata
+
+def test_plan_counts_pairs_and_rejects_bad_metadata(ba):
+    for kind in (W.CHAIN, W.BLOCK, W.TREE):
+        p = W.odd_shapes(kind)
+        assert ba.Plan(p).pairs == W.useful_pairs(p)
+    p = W.config1()
+    assert ba.Plan(p).pairs == 126184
+
+    def expect_meta_error(q):
+        with pytest.raises(ba.BranchAttnError) as e:
+            ba.Plan(q)
+        assert e.value.code == -4, e.value
+
+    import copy
+    q = copy.copy(W.odd_shapes(W.CHAIN)); q.anchor_idx = q.anchor_idx.copy(); q.anchor_idx[3] = 0
+    expect_meta_error(q)                                      # anchors not sorted
+    q = copy.copy(W.odd_shapes(W.CHAIN)); q.anchor_idx = q.anchor_idx.copy(); q.anchor_idx[-1] = 405
+    expect_meta_error(q)                                      # anchor == N
+    q = copy.copy(W.odd_shapes(W.TREE)); q.parent = q.parent.copy(); q.parent[5] = 7
+    expect_meta_error(q)                                      # parent[i] >= i
+    q = copy.copy(W.odd_shapes(W.CHAIN)); q.cu_seqlens = q.cu_seqlens.copy(); q.cu_seqlens[2] = 0
+    expect_meta_error(q)                                      # cu_seqlens decreasing
+    q = copy.copy(W.odd_shapes(W.BLOCK))
+    q.branch_offsets = np.array([0, 70] + [70 + 3 * i for i in range(1, 12)], dtype=np.int32)
+    expect_meta_error(q)                                      # a branch of 70 tokens
+    torch.cuda.synchronize()
+
+
+# --------------------------------------------------------------------- merge
+
+def test_lse_merge_matches_oracle(ba, oracle):
+    rng = np.random.default_rng(0)
+    rows, h, d = 1000, 3, 128
+    oa, ob = rng.standard_normal((2, rows, h, d)).astype(np.float32)
+    la, lb = (rng.standard_normal((2, rows, h)) * 5).astype(np.float32)
+    la[::7] = -np.inf
+    lb[::5] = -np.inf                                        # rows 0, 35, ... have both empty
+    lb[3] = la[3] + 60.0
+    want_o, want_l = oracle.lse_merge(oa, la, ob, lb)
+    toa, tob, tla, tlb = (torch.from_numpy(x).cuda() for x in (oa, ob, la, lb))
+    o, l = ba.lse_merge(toa, tla, tob, tlb)
+    assert_close("O", f32(o), want_o, 1e-5)
+    assert_lse_close(f32(l), want_l)
+    assert np.abs(f32(l)[~np.isneginf(want_l)] - want_l[~np.isneginf(want_l)]).max() < 1e-5
+    ob16, _ = ba.lse_merge(toa, tla, tob, tlb, out_dtype=torch.bfloat16)
+    assert_close("O bf16", f32(ob16), want_o, 2e-2)
+    # in place into (o_a, lse_a); d = 64 variant
+    oa64, ob64 = toa[..., :64].contiguous(), tob[..., :64].contiguous()
+    w_o, w_l = oracle.lse_merge(oa[..., :64], la, ob[..., :64], lb)
+    la_c = tla.clone()
+    ba.lse_merge(oa64, la_c, ob64, tlb, out=oa64, lse_out=la_c)
+    assert_close("O in place", f32(oa64), w_o, 1e-5)
+    assert_lse_close(f32(la_c), w_l)
+
+
+# ----------------------------------------------------------- the five configs
+
+def test_config1_tiny_fp32_full(ba, oracle):
+    check_full(ba, oracle, W.config1(), seed=0, std=1.0)
+
+
+@pytest.mark.parametrize("kind", [W.CHAIN, W.BLOCK, W.TREE])
+@pytest.mark.parametrize("dtype,d", [("fp32", 64), ("fp32", 128), ("bf16", 64), ("bf16", 128)])
+def test_odd_shapes_all_masks(ba, oracle, kind, dtype, d):
+    p = W.odd_shapes(kind, head_dim=d, dtype=dtype)
+    for impl in impls_for(ba, p):
+        check_full(ba, oracle, p, seed=3, std=1.0 if dtype == "fp32" else 0.5, impl=impl)
+
+
+@pytest.mark.parametrize("kind", [W.CHAIN, W.TREE])
+def test_branch_queries_only(ba, oracle, kind):
+    p = W.odd_shapes(kind, head_dim=128, dtype="bf16")
+    for impl in impls_for(ba, p):
+        check_full(ba, oracle, p, seed=4, std=0.5, impl=impl, q_main=False)
+
+
+@pytest.mark.parametrize("cfg,shrink", [(2, 8), (3, 16), (4, 16), (5, 128)])
+def test_shrunken_configs_bf16(ba, oracle, cfg, shrink):
+    p = W.CONFIGS[cfg](shrink)
+    for impl in impls_for(ba, p):
+        check_full(ba, oracle, p, seed=0, std=0.5, impl=impl, backward=(cfg != 2), groups=[0, p.h_kv - 1])
+
+
+def test_no_branches(ba, oracle):
+    cu = W.cu_from_lengths([100, 300, 29])
+    p = W.Problem(cu, np.zeros(0, np.int32), np.zeros(1, np.int32), W.CHAIN, None, 4, 2, 128, dtype="bf16")
+    for impl in impls_for(ba, p):
+        check_full(ba, oracle, p, seed=5, std=0.5, impl=impl)
+
+
+# ----------------------------------------------------------------- stress
+
+def _sharp(t):
+    t["q_main"] *= 8
+    t["q_branch"] *= 8
+
+
+def _offset(t):
+    rng = np.random.default_rng(99)
+    c = W.round_to_bf16(rng.standard_normal(t["k"].shape[-1]).astype(np.float32) * 4)
+    t["k"] += c
+    t["k"][:] = W.round_to_bf16(t["k"])
+
+
+def _late_outlier(t):
+    t["k"][400] = W.round_to_bf16(t["q_main"][404, 0] * 3)   # one key aligned with a late query
+
+
+@pytest.mark.parametrize("mutate", [_sharp, _offset, _late_outlier])
+def test_stress_inputs(ba, oracle, mutate):
+    p = W.odd_shapes(W.CHAIN, head_dim=128, dtype="bf16", h_q=4, h_kv=2)
+    for impl in impls_for(ba, p):
+        check_full(ba, oracle, p, seed=6, std=0.5, impl=impl, mutate=mutate)
+
+
+# ------------------------------------------------------- partial mode + merge
+
+@pytest.mark.parametrize("dtype,d", [("fp32", 64), ("bf16", 128)])
+def test_partial_chunks_merge_to_monolithic(ba, oracle, dtype, d):
+    p = W.odd_shapes(W.TREE, head_dim=d, dtype=dtype)
+    t = W.make_tensors(p, seed=7, std=0.5)
+    dv_ = to_dev(p, t)
+    n, a = p.n_main, p.num_branches
+    tol = TOL[dtype]
+    for impl in impls_for(ba, p):
+        plan = ba.Plan(p, impl=impl)
+        o_full, lse_full = ba.branch_attn_fwd(plan, dv_["q_main"], dv_["q_branch"], dv_["k"], dv_["v"])
+        # query block: main rows [10, 300), branches [2, 11); key chunks with ragged edges
+        qm, br = (10, 300), (2, 11)
+        t0, t1 = plan.token_range(*br)
+        rows = np.concatenate([np.arange(*qm), n + np.arange(t0, t1)])
+        chunks = [(0, 17), (17, 18), (18, 150), (150, 150), (150, n)]
+        acc = None
+        for i, kv in enumerate(chunks):
+            parts = ba.PART_MAIN | (ba.PART_BRANCH if i == 2 else 0)
+            o_p, l_p = ba.branch_attn_fwd_partial(plan, dv_["q_main"], dv_["q_branch"], dv_["k"], dv_["v"],
+                                                  qm, br, kv, parts)
+            ref = oracle_fwd_bwd(oracle, p, t, rows=rows, backward=False, parts=parts, kv_range=kv)
+            assert_close(f"O_part{i}", f32(o_p), ref["o"], tol)
+            assert_lse_close(f32(l_p), ref["lse"])
+            acc = (o_p, l_p) if acc is None else ba.lse_merge(acc[0], acc[1], o_p, l_p, out=acc[0], lse_out=acc[1])
+        rows_t = torch.from_numpy(rows).cuda()
+        assert_close("merged O", f32(acc[0]), f32(o_full[rows_t]).astype(np.float64), tol)
+        assert_lse_close(f32(acc[1]), f32(lse_full[rows_t]).astype(np.float64))
+
+        # backward: per-chunk accumulation equals the monolithic gradient
+        mono = ba.branch_attn_bwd(plan, dv_["q_main"], dv_["q_branch"], dv_["k"], dv_["v"], o_full, lse_full,
+                                  dv_["d_o"])
+        grads = None
+        for i, kv in enumerate(chunks):
+            parts = ba.PART_MAIN | (ba.PART_BRANCH if i == 2 else 0)
+            for qmr, brr in (((0, 100), (0, 5)), ((100, n), (5, a))):
+                grads = ba.branch_attn_bwd(plan, dv_["q_main"], dv_["q_branch"], dv_["k"], dv_["v"], o_full,
+                                           lse_full, dv_["d_o"], qm_range=qmr, br_range=brr, kv_range=kv,
+                                           parts=parts, accumulate=True, grads=grads)
+        ref = oracle_fwd_bwd(oracle, p, t)
+        want = (ref["dq"][:n], ref["dq"][n:], ref["dk"], ref["dv"])
+        for name, g_acc, g_mono, w in zip(("dQm", "dQb", "dK", "dV"), grads, mono, want):
+            assert_close(name + " accumulated", f32(g_acc), w, tol)
+            fin = ba.ba_finalize_grads(g_acc, dtype=plan.torch_dtype)
+            assert_close(name + " finalized", f32(fin), w, tol)
+            assert_close(name + " monolithic", f32(g_mono), w, tol)
+    torch.cuda.synchronize()
