@@ -36,6 +36,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 WORKLOADS = {
     "config5_256k_zigzag": (5, 1, 8, True),
     "config5_256k_monolithic": (5, 1, 0, True),
+    "config5_256k_zigzag_fwd": (5, 1, 8, False),
+    "config5_256k_monolithic_fwd": (5, 1, 0, False),
     "config5_64k_zigzag": (5, 4, 8, True),
     "config4_tree_64k": (4, 1, 0, True),
     "config3_dflash_32k": (3, 1, 0, True),

@@ -110,6 +110,11 @@ int64_t ba_plan_pairs(const ba_plan_t *plan);
 /* Which kernels the plan resolved to: BA_IMPL_SIMT or BA_IMPL_TC. */
 int ba_plan_impl(const ba_plan_t *plan);
 
+/* Synchronises `stream` and reports whether any kernel launched with this plan
+ * gave up a bounded device-side wait since the last check: BA_OK or BA_ETIMEOUT
+ * (the outputs of such a launch are undefined).  The flag is cleared. */
+int ba_plan_check(ba_plan_t *plan, void *stream);
+
 /*
  * Forward, both key sets fused in one online-softmax pass (Section 3.2: the
  * causal main-sequence component and the branch-local component; Eq.

@@ -44,7 +44,7 @@ class _Problem(C.Structure):
 
 _LIB = None
 EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
-           "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "branch_attn_fwd",
+           "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "ba_plan_check", "branch_attn_fwd",
            "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd", "ba_finalize_grads")
 
 
@@ -73,6 +73,8 @@ def _lib():
         lib.ba_plan_pairs.argtypes = [C.c_void_p]
         lib.ba_plan_impl.restype = C.c_int
         lib.ba_plan_impl.argtypes = [C.c_void_p]
+        lib.ba_plan_check.restype = C.c_int
+        lib.ba_plan_check.argtypes = [C.c_void_p, C.c_void_p]
         vp, i64 = C.c_void_p, C.c_int64
         lib.branch_attn_fwd.restype = C.c_int
         lib.branch_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
@@ -150,6 +152,10 @@ class Plan:
             n = _lib().ba_workspace_bytes(self.handle, op)
             self._ws[op] = torch.empty(max(n, 256), dtype=torch.uint8, device=self.device)
         return self._ws[op]
+
+    def check(self):
+        """Synchronise and raise if a kernel of this plan gave up a bounded wait."""
+        _check(_lib().ba_plan_check(self.handle, _stream()), "ba_plan_check")
 
     def close(self):
         if getattr(self, "handle", None):

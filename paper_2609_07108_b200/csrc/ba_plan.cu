@@ -310,3 +310,13 @@ extern "C" int ba_plan_destroy(ba_plan_t *plan) {
 extern "C" int64_t ba_plan_pairs(const ba_plan_t *plan) { return plan ? plan->pairs : -1; }
 
 extern "C" int ba_plan_impl(const ba_plan_t *plan) { return plan ? plan->impl : BA_EINVAL; }
+
+extern "C" int ba_plan_check(ba_plan_t *plan, void *stream) {
+    if (!plan) return BA_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t status = 0;
+    BA_CUDA_CHECK(cudaMemcpyAsync(&status, plan->dev_status, 4, cudaMemcpyDeviceToHost, st));
+    BA_CUDA_CHECK(cudaMemsetAsync(plan->dev_status, 0, 4, st));
+    BA_CUDA_CHECK(cudaStreamSynchronize(st));
+    return status == 0 ? BA_OK : BA_ETIMEOUT;
+}

@@ -1,15 +1,472 @@
-// Tensor-core (tcgen05) forward: placeholder until the kernels land.
+// Tensor-core forward (sm_100a, bf16, head_dim 128).
+//
+// One CTA = 128 query rows x two query heads of one KV head (both heads see the
+// same rows, hence the same key tiles and masks) -- or, when the group has an
+// odd head left over, that head twice with the second copy discarded.  Both
+// key sets of the paper's Section 3.2 (causal main prefix, own-branch keys) are
+// walked as 128-key tiles in ONE online-softmax pass, which is Eq. (lse-merge)
+// applied tile by tile; tiles no row can see are never visited, tiles every row
+// sees entirely take a mask-free path.
+//
+// Warp roles (320 threads):
+//   warps 0-3 / 4-7  softmax of query tile 0 / 1: one thread per row, scores read
+//                    from TMEM, P written back to TMEM as bf16 over the scores
+//   warp 8           issues tcgen05.mma: S_i = Q_i K^T, O_i += P_i V
+//   warp 9           TMA producer: Q once, then K_j, V_j through a 4-stage ring
+// The two query tiles ping-pong: while the softmax warps of tile 0 work on S_0,
+// the tensor core runs tile 1's P V and next Q K^T, and vice versa.
+// TMEM (512 columns): S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512);
+// P_i occupies the first 64 columns of S_i.
+#include <limits.h>
+#include <string.h>
+
 #include "ba_common.cuh"
+#include "ba_sm100.cuh"
 
-bool ba_tc_supported(const ba_problem_t *) { return false; }
+using namespace sm100;
 
-int ba_tc_fwd(const ba_plan *, const BaRange &, const void *, const void *, const void *, const void *,
-              void *, float *, bool, cudaStream_t) {
-    return BA_EUNSUPPORTED;
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kStages = 4;
+constexpr int kThreads = 320;
+constexpr uint32_t kTileBytes = 32768;  // 128 rows x 128 bf16
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;  // in log2 units: P stays below 2^8
+
+struct FwdSmem {
+    alignas(1024) uint8_t q[2][kTileBytes];
+    alignas(1024) uint8_t kv[kStages][kTileBytes];
+    alignas(8) uint64_t q_full;
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_full[2], p_full[2], o_full[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int lo_min, hi_max, lo_max, hi_min, bs_min, be_max;
+};
+
+struct TcFwdParams {
+    BaMeta meta;
+    BaRange r;
+    void *o;
+    float *lse;
+    int h_q, h_kv, group, pairs_per_group;
+    float scale_log2;
+    int partial_out;
+    int main_tiles, total_tiles;
+    int *status;
+};
+
+// bits [lo, hi] of a 64-bit word (empty if lo > hi)
+__device__ __forceinline__ uint64_t bit_range(int lo, int hi) {
+    lo = max(lo, 0);
+    hi = min(hi, 63);
+    if (lo > hi) return 0ull;
+    return (~0ull >> (63 - hi)) & (~0ull << lo);
 }
 
-int ba_tc_bwd(const ba_plan *, const BaRange &, const void *, const void *, const void *, const void *,
-              const float *, const float *, const void *, int, void *, void *, void *, void *,
-              cudaStream_t) {
-    return BA_EUNSUPPORTED;
+template <bool OUT_F32>
+__device__ __forceinline__ void store_row_chunk(void *o, size_t elem_off, const uint32_t (&r)[32], float inv) {
+    if (OUT_F32) {
+        float4 *dst = reinterpret_cast<float4 *>((float *)o + elem_off);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
+                                 __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
+    } else {
+        uint4 *dst = reinterpret_cast<uint4 *>((__nv_bfloat16 *)o + elem_off);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(r[8 * i]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
+            dst[i] = v;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constant__ CUtensorMap tm_q_branch,
+              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+              const TcFwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    FwdSmem &sm = *reinterpret_cast<FwdSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int *abort_flag = &sm.abort_flag;
+
+    // ---- work item: later (longer-prefix) row tiles first; the CTAs of one row
+    // tile (all KV heads and head pairs) are adjacent so they share K/V in L2
+    const int per_tile = p.h_kv * p.pairs_per_group;
+    const int tile = p.total_tiles - 1 - (int)(blockIdx.x / per_tile);
+    const int inner = (int)(blockIdx.x % per_tile);
+    const int g = inner / p.pairs_per_group, hp = inner % p.pairs_per_group;
+    const int h0 = g * p.group + 2 * hp;
+    const bool second_head = 2 * hp + 1 < p.group;
+    const int h1 = second_head ? h0 + 1 : h0;
+    const bool is_main = tile < p.main_tiles;
+    const int64_t n = p.meta.n_main;
+    // first row of the tile inside its tensor (q_main rows / q_branch tokens)
+    const int64_t row0 = is_main ? p.r.qm_begin + (int64_t)tile * kTile
+                                 : p.r.tok_begin + (int64_t)(tile - p.main_tiles) * kTile;
+    const int64_t row_end = is_main ? p.r.qm_end : p.r.tok_end;
+
+    if (tid == 0) {
+        mbar_init(&sm.q_full, 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sm.s_full[i], 1);
+            mbar_init(&sm.p_full[i], 128);
+            mbar_init(&sm.o_full[i], 1);
+        }
+        sm.abort_flag = 0;
+        sm.lo_min = INT_MAX; sm.hi_max = -1; sm.lo_max = -1; sm.hi_min = INT_MAX;
+        sm.bs_min = INT_MAX; sm.be_max = -1;
+        fence_barrier_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(&sm.tmem_base, 512);
+        tmem_relinquish();
+    }
+    if (warp == 9 && lane == 0) {
+        tma_prefetch_desc(is_main ? &tm_q_main : &tm_q_branch);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    __syncthreads();
+
+    // ---- per-row metadata (softmax threads: row = tid % 128)
+    int lo = 1, hi = 0, bstart = 0;
+    uint64_t bmask = 0;
+    bool valid = false;
+    int64_t my_row = 0;
+    if (warp < 8) {
+        my_row = row0 + (tid & 127);
+        valid = my_row < row_end;
+        if (valid) {
+            const int64_t grow = is_main ? my_row : n + my_row;
+            if (p.r.parts & BA_PART_MAIN) {
+                lo = max(p.meta.row_lo[grow], (int)p.r.kv_begin);
+                hi = min(p.meta.row_hi[grow], (int)p.r.kv_end - 1);
+                if (hi < lo) { lo = 1; hi = 0; }
+            }
+            if (!is_main && (p.r.parts & BA_PART_BRANCH)) {
+                bstart = p.meta.br_start[my_row];
+                bmask = p.meta.br_mask[my_row];
+            }
+            if (warp < 4) {
+                if (hi >= lo) {
+                    atomicMin(&sm.lo_min, lo); atomicMax(&sm.hi_max, hi);
+                    atomicMax(&sm.lo_max, lo); atomicMin(&sm.hi_min, hi);
+                } else {
+                    atomicMax(&sm.lo_max, INT_MAX); atomicMin(&sm.hi_min, -1);
+                }
+                if (!is_main && (p.r.parts & BA_PART_BRANCH)) {
+                    atomicMin(&sm.bs_min, bstart);
+                    atomicMax(&sm.be_max, p.meta.br_end[my_row]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    // ---- key tiles: aligned 128-key main tiles [kt0, kt0 + n_main), then the
+    // own-branch keys [bs, be) as n_br tiles starting at bs
+    int kt0 = 0, n_main_tiles = 0, n_br = 0;
+    if (sm.hi_max >= sm.lo_min) {
+        kt0 = sm.lo_min / kTile;
+        n_main_tiles = sm.hi_max / kTile - kt0 + 1;
+    }
+    const int bs = sm.bs_min;
+    if (sm.be_max > bs) n_br = (sm.be_max - bs + kTile - 1) / kTile;
+    const int T = n_main_tiles + n_br;
+    const int full_lo = sm.lo_max, full_hi = sm.hi_min;
+
+    if (warp == 9) {
+        // ================================================= TMA producer
+        if (lane == 0 && T > 0) {
+            const CUtensorMap *tq = is_main ? &tm_q_main : &tm_q_branch;
+            mbar_expect_tx(&sm.q_full, 2 * kTileBytes);
+            for (int half = 0; half < 2; ++half) {
+                tma_load_3d(sm.q[0] + half * 16384, tq, half * 64, h0, (int)row0, &sm.q_full);
+                tma_load_3d(sm.q[1] + half * 16384, tq, half * 64, h1, (int)row0, &sm.q_full);
+            }
+            int issued = 0;
+            bool ok = true;
+            for (int it = 0; it < 2 * T && ok; ++it) {
+                const int j = it >> 1, s = it % kStages;
+                if (it >= kStages) ok = mbar_wait(&sm.kv_empty[s], ((it / kStages) - 1) & 1, abort_flag);
+                if (!ok) break;
+                const int krow = j < n_main_tiles ? (kt0 + j) * kTile
+                                                  : (int)n + bs + (j - n_main_tiles) * kTile;
+                const CUtensorMap *tkv = (it & 1) ? &tm_v : &tm_k;
+                mbar_expect_tx(&sm.kv_full[s], kTileBytes);
+                tma_load_3d(sm.kv[s], tkv, 0, g, krow, &sm.kv_full[s]);
+                tma_load_3d(sm.kv[s] + 16384, tkv, 64, g, krow, &sm.kv_full[s]);
+                issued = it + 1;
+            }
+            if (!ok) {
+                // leave no copy in flight behind: wait (bounded) for what was issued
+                for (int it = max(issued - kStages, 0); it < issued; ++it) {
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(&sm.kv_full[it % kStages], (it / kStages) & 1) && ++spins < (1u << 22)) {}
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ================================================= MMA issuer
+        if (lane == 0 && T > 0) {
+            constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, 0);
+            constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, 1);
+            const uint32_t q_addr[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
+            auto issue_qk = [&](int i, int stage) {
+                const uint32_t k_addr = smem_u32(sm.kv[stage]);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+                    mma_ss(tmem + i * 128, smem_desc_sw128(q_addr[i] + off, 16, 1024),
+                           smem_desc_sw128(k_addr + off, 16, 1024), IDESC_QK, ks > 0);
+                }
+            };
+            auto issue_pv = [&](int i, int stage, bool accumulate) {
+                const uint32_t v_addr = smem_u32(sm.kv[stage]);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(tmem + 256 + i * 128, tmem + i * 128 + ks * 8,
+                           smem_desc_sw128(v_addr + ks * 2048, 16384, 1024), IDESC_PV, accumulate || ks > 0);
+            };
+            bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
+            ok = ok && mbar_wait(&sm.kv_full[0], 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0, 0); tc_commit(&sm.s_full[0]);
+                issue_qk(1, 0); tc_commit(&sm.s_full[1]);
+                tc_commit(&sm.kv_empty[0]);
+            }
+            for (int j = 0; j < T && ok; ++j) {
+                const int it_v = 2 * j + 1, sv = it_v % kStages;
+                const int it_k = 2 * j + 2, sk = it_k % kStages;
+                for (int i = 0; i < 2 && ok; ++i) {
+                    ok = mbar_wait(&sm.p_full[i], j & 1, abort_flag);
+                    if (ok && i == 0) ok = mbar_wait(&sm.kv_full[sv], (it_v / kStages) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(i, sv, j > 0);
+                    if (i == 1) tc_commit(&sm.kv_empty[sv]);
+                    if (j + 1 < T) {
+                        if (i == 0) {
+                            ok = mbar_wait(&sm.kv_full[sk], (it_k / kStages) & 1, abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        issue_qk(i, sk); tc_commit(&sm.s_full[i]);
+                        if (i == 1) tc_commit(&sm.kv_empty[sk]);
+                    } else {
+                        tc_commit(&sm.o_full[i]);
+                    }
+                }
+            }
+        }
+    } else {
+        // ================================================= softmax + epilogue
+        const int i = warp >> 2;                                   // query tile 0 / 1
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t s_addr = tmem + lane_base + i * 128;
+        const uint32_t o_addr = tmem + lane_base + 256 + i * 128;
+        const float sl2 = p.scale_log2;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < T; ++j) {
+            ok = mbar_wait(&sm.s_full[i], j & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            // --- visibility of this tile's 128 key columns for my row
+            bool masked;
+            uint64_t vis[2] = {~0ull, ~0ull};
+            if (j < n_main_tiles) {
+                const int kj = (kt0 + j) * kTile;
+                masked = !(kj >= full_lo && kj + kTile - 1 <= full_hi);
+                if (masked) {
+                    vis[0] = bit_range(lo - kj, hi - kj);
+                    vis[1] = bit_range(lo - kj - 64, hi - kj - 64);
+                }
+            } else {
+                masked = true;
+                // column c is branch token bs + 128 (j - n_main_tiles) + c; bit c = bmask bit (c + off)
+                const int off = bs + (j - n_main_tiles) * kTile - bstart;
+                const uint64_t mk = valid ? bmask : 0ull;
+                if (off >= 0) {
+                    vis[0] = off < 64 ? mk >> off : 0ull;
+                    vis[1] = 0ull;
+                } else {
+                    const int sh = -off;
+                    if (sh < 64) { vis[0] = mk << sh; vis[1] = mk >> (64 - sh); }
+                    else if (sh < 128) { vis[0] = 0ull; vis[1] = mk << (sh - 64); }
+                    else { vis[0] = 0ull; vis[1] = 0ull; }
+                }
+            }
+            // --- pass 1: row maximum
+            float m_tile = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(s_addr + c * 32, r);
+                tmem_wait_ld();
+                if (masked) {
+                    const uint32_t mk = (uint32_t)(vis[c >> 1] >> ((c & 1) * 32));
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        m_tile = fmaxf(m_tile, ((mk >> e) & 1u) ? __uint_as_float(r[e]) : -INFINITY);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) m_tile = fmaxf(m_tile, __uint_as_float(r[e]));
+                }
+            }
+            // --- running maximum; O and l are rescaled only when it grew a lot
+            const float m_new = fmaxf(m_run, m_tile);
+            float alpha = 1.0f;
+            const bool grow = m_new > m_run && (m_run == -INFINITY || (m_new - m_run) * sl2 > kRescaleThreshold);
+            if (grow) {
+                alpha = exp2f((m_run - m_new) * sl2);  // m_run = -inf gives 0
+                l_run *= alpha;
+                m_run = m_new;
+            }
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(o_addr + c * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                    tmem_st32(o_addr + c * 32, r);
+                }
+            }
+            const float neg_ms = m_run == -INFINITY ? 0.f : -m_run * sl2;
+            // --- pass 2: P = exp2(s * scale_log2 - m), bf16, over the first 64 score columns
+            float l_add = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32], pk[16];
+                tmem_ld32(s_addr + c * 32, r);
+                tmem_wait_ld();
+                const uint32_t mk = masked ? (uint32_t)(vis[c >> 1] >> ((c & 1) * 32)) : 0xffffffffu;
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float p0 = exp2f(fmaf(__uint_as_float(r[e]), sl2, neg_ms));
+                    float p1 = exp2f(fmaf(__uint_as_float(r[e + 1]), sl2, neg_ms));
+                    if (masked) {
+                        p0 = ((mk >> e) & 1u) ? p0 : 0.f;
+                        p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
+                    }
+                    l_add += p0 + p1;
+                    pk[e >> 1] = pack_bf16(p0, p1);
+                }
+                tmem_st16(s_addr + c * 16, pk);
+            }
+            l_run += l_add;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm.p_full[i]);
+        }
+        // --- epilogue: O / l and LSE
+        if (ok && T > 0) ok = mbar_wait(&sm.o_full[i], 0, abort_flag);
+        tc_fence_after();
+        {
+            const bool do_store = ok && valid && (i == 0 || second_head);
+            const int h = i == 0 ? h0 : h1;
+            int64_t orow = is_main ? my_row : n + my_row;
+            if (p.partial_out)
+                orow = is_main ? my_row - p.r.qm_begin : (p.r.qm_end - p.r.qm_begin) + (my_row - p.r.tok_begin);
+            const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
+            const size_t base = ((size_t)orow * p.h_q + h) * 128;
+            if (do_store)
+                p.lse[orow * p.h_q + h] = l_run > 0.f ? (m_run * sl2 + log2f(l_run)) * kLn2 : -INFINITY;
+            // every lane runs the (warp-collective) TMEM loads; only live rows store
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                if (T > 0 && ok) {
+                    tmem_ld32(o_addr + c * 32, r);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
+                if (do_store) {
+                    if (p.partial_out) store_row_chunk<true>(p.o, base + c * 32, r, inv);
+                    else store_row_chunk<false>(p.o, base + c * 32, r, inv);
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (tid == 0 && sm.abort_flag) atomicExch(p.status, BA_ETIMEOUT);
+}
+
+}  // namespace
+
+bool ba_tc_supported(const ba_problem_t *p) {
+    return p->dtype == BA_BF16 && p->head_dim == 128 && encode_tiled_fn() != nullptr;
+}
+
+int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
+              const void *v, void *o, float *lse, bool partial_out, cudaStream_t st) {
+    static bool attr_set = false;
+    const size_t smem = sizeof(FwdSmem) + 1024;
+    if (!attr_set) {
+        BA_CUDA_CHECK(cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set = true;
+    }
+    const ba_problem_t &pr = pl->prob;
+    TcFwdParams p;
+    memset(&p, 0, sizeof p);
+    p.meta = pl->meta;
+    p.r = r;
+    p.o = o;
+    p.lse = lse;
+    p.h_q = pr.h_q;
+    p.h_kv = pr.h_kv;
+    p.group = pr.h_q / pr.h_kv;
+    p.pairs_per_group = (p.group + 1) / 2;
+    p.scale_log2 = pl->scale * kLog2e;
+    p.partial_out = partial_out ? 1 : 0;
+    p.status = pl->dev_status;
+    const int64_t mt = q_main ? (r.qm_end - r.qm_begin + kTile - 1) / kTile : 0;
+    const int64_t bt = (r.tok_end - r.tok_begin + kTile - 1) / kTile;
+    p.main_tiles = (int)mt;
+    p.total_tiles = (int)(mt + bt);
+    if (p.total_tiles == 0) return BA_OK;
+
+    CUtensorMap tq_main, tq_branch, tk, tv;
+    const uint64_t kv_rows = (uint64_t)(pr.n_main + pr.n_branch);
+    if (!make_tmap_rhd(&tk, k, kv_rows, pr.h_kv, 128, kTile) || !make_tmap_rhd(&tv, v, kv_rows, pr.h_kv, 128, kTile))
+        return BA_EINVAL;
+    // an absent query tensor still needs a valid map object: alias the other one
+    const void *qm = q_main ? q_main : q_branch;
+    const void *qb = (q_branch && pr.n_branch > 0) ? q_branch : q_main;
+    const uint64_t qm_rows = q_main ? (uint64_t)pr.n_main : (uint64_t)pr.n_branch;
+    const uint64_t qb_rows = (q_branch && pr.n_branch > 0) ? (uint64_t)pr.n_branch : (uint64_t)pr.n_main;
+    if (!make_tmap_rhd(&tq_main, qm, qm_rows, pr.h_q, 128, kTile) ||
+        !make_tmap_rhd(&tq_branch, qb, qb_rows, pr.h_q, 128, kTile))
+        return BA_EINVAL;
+    const int64_t grid = (int64_t)p.total_tiles * pr.h_kv * p.pairs_per_group;
+    if (grid > INT_MAX) return BA_EUNSUPPORTED;
+    tc_fwd_kernel<<<(unsigned)grid, kThreads, smem, st>>>(tq_main, tq_branch, tk, tv, p);
+    return ba_check_launch();
+}
+
+int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
+              const void *v, const float *lse, const float *delta, const void *d_o, int accumulate,
+              void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st) {
+    // tensor-core backward kernels are not in yet: the plain-FMA kernels do it
+    return ba_simt_bwd(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, dq_main, dq_branch, dk, dv, st);
 }

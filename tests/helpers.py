@@ -35,6 +35,9 @@ def head_slice(p, groups):
 
 def assert_close(name, got, want, tol):
     got = np.asarray(got, dtype=np.float64)
+    assert got.shape == np.shape(want), f"{name}: shape {got.shape} vs {np.shape(want)}"
+    if got.size == 0:
+        return
     err = np.abs(got - want)
     assert np.isfinite(got).all(), f"{name}: non-finite values"
     assert err.max() <= tol, f"{name}: max abs err {err.max():.3e} > {tol:.1e} at {np.unravel_index(err.argmax(), err.shape)}"

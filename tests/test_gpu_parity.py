@@ -36,6 +36,7 @@ def check_full(ba, oracle, p, seed=0, std=1.0, impl=None, backward=True, groups=
     n = p.n_main
     qm = d["q_main"] if q_main else None
     o, lse = ba.branch_attn_fwd(plan, qm, d["q_branch"], d["k"], d["v"])
+    plan.check()
     ref = oracle_fwd_bwd(oracle, p, t, groups=groups, backward=backward)
     qh, kvh = ref["q_heads"], ref["kv_heads"]
     tol = TOL[p.dtype]
@@ -56,7 +57,7 @@ def check_full(ba, oracle, p, seed=0, std=1.0, impl=None, backward=True, groups=
     assert_close("dQ_branch", f32(dqb)[:, qh], ref["dq"][n:], tol)
     assert_close("dK", f32(dk)[:, kvh], ref["dk"], tol)
     assert_close("dV", f32(dv)[:, kvh], ref["dv"], tol)
-    torch.cuda.synchronize()
+    plan.check()
 
 
 # ------------------------------------------------------------------ metadata
