@@ -423,9 +423,9 @@ int launch_fwd(SimtArgs &a, cudaStream_t st) {
 }
 
 template <typename T, int D>
-int launch_bwd(SimtArgs &a, cudaStream_t st) {
+int launch_bwd(SimtArgs &a, cudaStream_t st, bool do_dq, bool do_dkdv) {
     constexpr int RB = kThreads / (D / 32);
-    {
+    if (do_dq) {
         const int64_t mt = a.q_main ? ceil_div(a.r.qm_end - a.r.qm_begin, RB) : 0;
         const int64_t bt = ceil_div(a.r.tok_end - a.r.tok_begin, RB);
         a.main_tiles = mt;
@@ -436,7 +436,7 @@ int launch_bwd(SimtArgs &a, cudaStream_t st) {
             if (rc != BA_OK) return rc;
         }
     }
-    {
+    if (do_dkdv) {
         const int64_t mt = (a.r.parts & BA_PART_MAIN) ? ceil_div(a.r.kv_end - a.r.kv_begin, RB) : 0;
         const int64_t bt = (a.r.parts & BA_PART_BRANCH) ? ceil_div(a.r.tok_end - a.r.tok_begin, RB) : 0;
         a.main_tiles = mt;
@@ -448,6 +448,21 @@ int launch_bwd(SimtArgs &a, cudaStream_t st) {
         }
     }
     return BA_OK;
+}
+
+int bwd_dispatch(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
+                 const void *k, const void *v, const float *lse, const float *delta, const void *d_o,
+                 int accumulate, void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st,
+                 bool do_dq, bool do_dkdv) {
+    SimtArgs a = base_args(pl, r);
+    a.q_main = q_main; a.q_branch = q_branch; a.k = k; a.v = v; a.d_o = d_o;
+    a.lse_in = lse; a.delta = delta; a.accumulate = accumulate;
+    a.dq_main = dq_main; a.dq_branch = dq_branch; a.dk = dk; a.dv = dv;
+    const int d = pl->prob.head_dim;
+    if (pl->prob.dtype == BA_FP32)
+        return d == 64 ? launch_bwd<float, 64>(a, st, do_dq, do_dkdv) : launch_bwd<float, 128>(a, st, do_dq, do_dkdv);
+    return d == 64 ? launch_bwd<__nv_bfloat16, 64>(a, st, do_dq, do_dkdv)
+                   : launch_bwd<__nv_bfloat16, 128>(a, st, do_dq, do_dkdv);
 }
 
 }  // namespace
@@ -467,11 +482,13 @@ int ba_simt_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const v
                 const void *k, const void *v, const float *lse, const float *delta,
                 const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
                 void *dv, cudaStream_t st) {
-    SimtArgs a = base_args(pl, r);
-    a.q_main = q_main; a.q_branch = q_branch; a.k = k; a.v = v; a.d_o = d_o;
-    a.lse_in = lse; a.delta = delta; a.accumulate = accumulate;
-    a.dq_main = dq_main; a.dq_branch = dq_branch; a.dk = dk; a.dv = dv;
-    const int d = pl->prob.head_dim;
-    if (pl->prob.dtype == BA_FP32) return d == 64 ? launch_bwd<float, 64>(a, st) : launch_bwd<float, 128>(a, st);
-    return d == 64 ? launch_bwd<__nv_bfloat16, 64>(a, st) : launch_bwd<__nv_bfloat16, 128>(a, st);
+    return bwd_dispatch(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, dq_main, dq_branch, dk, dv,
+                        st, true, true);
+}
+
+int ba_simt_bwd_dkdv(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
+                     const void *k, const void *v, const float *lse, const float *delta,
+                     const void *d_o, int accumulate, void *dk, void *dv, cudaStream_t st) {
+    return bwd_dispatch(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, nullptr, nullptr, dk, dv,
+                        st, false, true);
 }

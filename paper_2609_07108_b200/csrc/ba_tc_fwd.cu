@@ -463,10 +463,3 @@ int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
     tc_fwd_kernel<<<(unsigned)grid, kThreads, smem, st>>>(tq_main, tq_branch, tk, tv, p);
     return ba_check_launch();
 }
-
-int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
-              const void *v, const float *lse, const float *delta, const void *d_o, int accumulate,
-              void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st) {
-    // tensor-core backward kernels are not in yet: the plain-FMA kernels do it
-    return ba_simt_bwd(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, dq_main, dq_branch, dk, dv, st);
-}
