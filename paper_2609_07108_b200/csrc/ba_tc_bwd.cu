@@ -399,6 +399,368 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
     if (tid == 0 && sm.abort_flag) atomicExch(p.status, BA_ETIMEOUT);
 }
 
+
+// ============================================================================
+// dK / dV
+// ============================================================================
+// Key-stationary: one CTA owns 128 key rows of one KV head, keeps K_j, V_j in
+// shared memory and dK_j, dV_j (fp32) in TMEM, and walks the query rows that
+// can see those keys -- all query heads of the KV head -- as 64-row sub-tiles.
+// Everything is computed transposed so that the key index is the TMEM lane:
+//   S^T = K_j Q^T, dP^T = V_j dO^T        (128 keys x 64 query rows)
+//   P^T = exp2(scale_log2 S^T - lse2[col]),  dS^T = P^T o (dP^T - delta[col])
+//   dV_j += P^T dO,  dK_j += dS^T Q          (P^T, dS^T are TMEM A operands)
+// Two sub-tiles are in flight (sets 0 / 1, one softmax warpgroup each).
+//   TMEM: dK [0,128) dV [128,256); set b: X_b = 256 + 128 b (64 cols: S^T, then
+//   dP^T), Y_b = X_b + 64 (P^T in cols [0,32), dS^T in cols [32,64))
+constexpr int kKvThreads = 320;
+constexpr int kSub = 64;           // query rows per sub-tile
+constexpr int kQStages = 4;
+constexpr uint32_t kSubBytes = 16384;  // 64 rows x 128 bf16
+
+struct SubMeta {
+    float neg_lse2[kSub];
+    float delta[kSub];
+    int bstart[kSub];
+    unsigned long long mask[kSub];
+};
+
+struct KvSmem {
+    alignas(1024) uint8_t k[kTileBytes];
+    alignas(1024) uint8_t v[kTileBytes];
+    alignas(1024) uint8_t qs[kQStages][2 * kSubBytes];  // Q sub-tile, then dO sub-tile
+    alignas(16) SubMeta meta[kQStages];
+    alignas(8) uint64_t kv_full;
+    uint64_t q_full[kQStages], q_empty[kQStages];
+    uint64_t s_full[2], a_done[2], dp_full[2], b_done[2], acc_full;
+    uint32_t tmem_base;
+    int abort_flag;
+    int qend_max, bq0_min, bq1_max;
+};
+
+__global__ void __launch_bounds__(kKvThreads, 1)
+tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constant__ CUtensorMap tm_q_branch,
+               const __grid_constant__ CUtensorMap tm_go, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const TcBwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    KvSmem &sm = *reinterpret_cast<KvSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    volatile int *abort_flag = &sm.abort_flag;
+
+    const int tile = (int)(blockIdx.x / p.h_kv);
+    const int g = (int)(blockIdx.x % p.h_kv);
+    const bool main_keys = tile < p.main_key_tiles;
+    const int64_t n = p.meta.n_main;
+    // first key of the tile: main key index, or branch token index
+    const int64_t key0 = main_keys ? p.r.kv_begin + (int64_t)tile * kTile
+                                   : p.r.tok_begin + (int64_t)(tile - p.main_key_tiles) * kTile;
+    const int64_t key_end = main_keys ? p.r.kv_end : p.r.tok_end;
+    const int64_t gkey0 = main_keys ? key0 : n + key0;
+
+    if (tid == 0) {
+        mbar_init(&sm.kv_full, 1);
+        for (int s = 0; s < kQStages; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.s_full[b], 1);
+            mbar_init(&sm.a_done[b], 128);
+            mbar_init(&sm.dp_full[b], 1);
+            mbar_init(&sm.b_done[b], 128);
+        }
+        mbar_init(&sm.acc_full, 1);
+        sm.abort_flag = 0;
+        sm.qend_max = -1; sm.bq0_min = INT_MAX; sm.bq1_max = -1;
+        fence_barrier_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(&sm.tmem_base, 512);
+        tmem_relinquish();
+    }
+    __syncthreads();
+
+    // ---- my key row (threads of both warpgroups: key = tid % 128)
+    bool kvalid = false;
+    int my_key = 0, my_qend = 0, my_bq0 = 0, my_bq1 = 0;
+    if (warp < 8) {
+        const int64_t kk = key0 + (tid & 127);
+        kvalid = kk < key_end;
+        my_key = (int)kk;
+        if (kvalid) {
+            if (main_keys) {
+                my_qend = p.meta.key_qend[kk];
+                my_bq0 = p.meta.key_bq_begin[kk];
+                my_bq1 = p.meta.key_bq_end[kk];
+            } else {
+                my_bq0 = p.meta.br_start[kk];
+                my_bq1 = p.meta.br_end[kk];
+            }
+            if (warp < 4) {
+                if (main_keys) atomicMax(&sm.qend_max, my_qend);
+                atomicMin(&sm.bq0_min, my_bq0);
+                atomicMax(&sm.bq1_max, my_bq1);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    // ---- query segments: main rows [m0, m1), branch tokens [b0, b1)
+    int64_t m0 = 0, m1 = 0, b0 = 0, b1 = 0;
+    if (main_keys && p.has_main_q) {
+        m0 = max(key0, p.r.qm_begin);
+        m1 = min((int64_t)sm.qend_max, p.r.qm_end);
+    }
+    if (sm.bq1_max > sm.bq0_min) {
+        b0 = max((int64_t)sm.bq0_min, p.r.tok_begin);
+        b1 = min((int64_t)sm.bq1_max, p.r.tok_end);
+    }
+    const int n_sub_main = m1 > m0 ? (int)((m1 - m0 + kSub - 1) / kSub) : 0;
+    const int n_sub_br = b1 > b0 ? (int)((b1 - b0 + kSub - 1) / kSub) : 0;
+    const int n_sub = n_sub_main + n_sub_br;
+    const int n_iter = n_sub * p.group;
+
+    if (warp == 9) {
+        // ================================================= producer (whole warp)
+        if (n_iter > 0) {
+            if (lane == 0) {
+                mbar_expect_tx(&sm.kv_full, 2 * kTileBytes);
+                for (int half = 0; half < 2; ++half) {
+                    tma_load_3d(sm.k + half * 16384, &tm_k, half * 64, g, (int)gkey0, &sm.kv_full);
+                    tma_load_3d(sm.v + half * 16384, &tm_v, half * 64, g, (int)gkey0, &sm.kv_full);
+                }
+            }
+            bool ok = true;
+            int issued = 0;
+            for (int t = 0; t < n_iter; ++t) {
+                const int st = t % kQStages;
+                if (t >= kQStages) ok = mbar_wait(&sm.q_empty[st], ((t / kQStages) - 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const int h = g * p.group + t / n_sub;
+                const int s = t % n_sub;
+                const bool seg_main = s < n_sub_main;
+                const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
+                const int64_t rend = seg_main ? m1 : b1;
+                const int64_t grow0 = seg_main ? r0 : n + r0;
+                SubMeta &mt = sm.meta[st];
+                for (int c = lane; c < kSub; c += 32) {
+                    const bool live = r0 + c < rend;
+                    mt.neg_lse2[c] = live ? -p.lse[(grow0 + c) * p.h_q + h] * kLog2e : -INFINITY;
+                    mt.delta[c] = live ? p.delta[(grow0 + c) * p.h_q + h] : 0.f;
+                    if (!main_keys) {
+                        mt.bstart[c] = live ? p.meta.br_start[r0 + c] : 0;
+                        mt.mask[c] = live ? p.meta.br_mask[r0 + c] : 0ull;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    const CUtensorMap *tq = seg_main ? &tm_q_main : &tm_q_branch;
+                    mbar_expect_tx(&sm.q_full[st], 2 * kSubBytes);
+                    for (int half = 0; half < 2; ++half) {
+                        tma_load_3d(sm.qs[st] + half * 8192, tq, half * 64, h, (int)r0, &sm.q_full[st]);
+                        tma_load_3d(sm.qs[st] + kSubBytes + half * 8192, &tm_go, half * 64, h, (int)grow0,
+                                    &sm.q_full[st]);
+                    }
+                }
+                issued = t + 1;
+            }
+            if (!ok && lane == 0) {
+                for (int t = max(issued - kQStages, 0); t < issued; ++t) {
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(&sm.q_full[t % kQStages], (t / kQStages) & 1) && ++spins < (1u << 22)) {}
+                }
+                uint32_t spins = 0;
+                while (!mbar_try_wait(&sm.kv_full, 0) && ++spins < (1u << 22)) {}
+            }
+        }
+    } else if (warp == 8) {
+        // ================================================= MMA issuer
+        if (lane == 0 && n_iter > 0) {
+            constexpr uint32_t IDESC_T = idesc_bf16(128, kSub, 0);   // 128 keys x 64 rows, K = d
+            constexpr uint32_t IDESC_ACC = idesc_bf16(128, 128, 1);  // 128 keys x 128 d, K = 64 rows
+            const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v);
+            auto issue_t = [&](uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ss(d_tmem, smem_desc_sw128(a_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                           smem_desc_sw128(b_addr + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), IDESC_T, ks > 0);
+            };
+            auto issue_acc = [&](uint32_t d_tmem, uint32_t a_tmem, uint32_t b_addr, bool accumulate) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ts(d_tmem, a_tmem + ks * 8, smem_desc_sw128(b_addr + ks * 2048, 8192, 1024), IDESC_ACC,
+                           accumulate || ks > 0);
+            };
+            bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
+            for (int b = 0; b < 2 && ok; ++b) {
+                if (b >= n_iter) break;
+                ok = mbar_wait(&sm.q_full[b], 0, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                issue_t(tmem + 256 + b * 128, k_addr, smem_u32(sm.qs[b]));
+                tc_commit(&sm.s_full[b]);
+            }
+            for (int t0 = 0; t0 < n_iter && ok; t0 += 2) {
+                for (int b = 0; b < 2 && ok; ++b) {
+                    const int t = t0 + b;
+                    if (t >= n_iter) break;
+                    const uint32_t stage_addr = smem_u32(sm.qs[t % kQStages]);
+                    ok = mbar_wait(&sm.a_done[b], (t >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_t(tmem + 256 + b * 128, v_addr, stage_addr + kSubBytes);     // dP^T = V dO^T
+                    tc_commit(&sm.dp_full[b]);
+                    issue_acc(tmem + 128, tmem + 256 + b * 128 + 64, stage_addr + kSubBytes, t > 0);  // dV += P^T dO
+                }
+                for (int b = 0; b < 2 && ok; ++b) {
+                    const int t = t0 + b;
+                    if (t >= n_iter) break;
+                    const uint32_t stage_addr = smem_u32(sm.qs[t % kQStages]);
+                    ok = mbar_wait(&sm.b_done[b], (t >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_acc(tmem + 0, tmem + 256 + b * 128 + 96, stage_addr, t > 0);                // dK += dS^T Q
+                    tc_commit(&sm.q_empty[t % kQStages]);
+                    const int t2 = t + 2;
+                    if (t2 < n_iter) {
+                        ok = mbar_wait(&sm.q_full[t2 % kQStages], (t2 / kQStages) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_t(tmem + 256 + b * 128, k_addr, smem_u32(sm.qs[t2 % kQStages]));
+                        tc_commit(&sm.s_full[b]);
+                    }
+                }
+            }
+            if (ok) tc_commit(&sm.acc_full);
+        }
+    } else {
+        // ================================================= P^T / dS^T warps + epilogue
+        const int b = warp >> 2;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t x_addr = tmem + lane_base + 256 + b * 128;
+        const uint32_t y_addr = x_addr + 64;
+        const float sl2 = p.scale_log2;
+        bool ok = true;
+        for (int t = b; t < n_iter; t += 2) {
+            const int st = t % kQStages;
+            const int s = t % n_sub;
+            const bool seg_main = s < n_sub_main;
+            const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
+            const int64_t rend = seg_main ? m1 : b1;
+            const SubMeta &mt = sm.meta[st];
+            ok = mbar_wait(&sm.s_full[b], (t >> 1) & 1, abort_flag);
+            ok = ok && mbar_wait(&sm.q_full[st], (t / kQStages) & 1, abort_flag);  // metadata of the stage
+            if (!ok) break;
+            tc_fence_after();
+            // --- which of the 64 query rows (columns) see my key
+            uint64_t vis = 0ull;
+            if (kvalid) {
+                if (main_keys) {
+                    if (seg_main)  // same sequence, causal: key <= row < end of the key's sequence
+                        vis = bit_range((int)(my_key - r0), (int)(min((int64_t)my_qend, rend) - 1 - r0));
+                    else           // branch tokens anchored at or after the key, inside its sequence
+                        vis = bit_range((int)(my_bq0 - r0), (int)(min((int64_t)my_bq1, rend) - 1 - r0));
+                } else {
+                    // own-branch tokens whose mask has my bit
+                    const int lo_c = max((int)(my_bq0 - r0), 0), hi_c = min((int)(min((int64_t)my_bq1, rend) - 1 - r0), kSub - 1);
+                    for (int c = lo_c; c <= hi_c; ++c) {
+                        const int rel = my_key - mt.bstart[c];
+                        if (rel >= 0 && rel < 64 && ((mt.mask[c] >> rel) & 1ull)) vis |= 1ull << c;
+                    }
+                }
+            }
+            const bool masked = !__all_sync(0xffffffffu, vis == ~0ull);
+            // --- phase A: P^T
+            uint32_t pr[32];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t r[32], pk[16];
+                tmem_ld32(x_addr + c * 32, r);
+                tmem_wait_ld();
+                const uint32_t mk = masked ? (uint32_t)(vis >> (c * 32)) : 0xffffffffu;
+                const float4 *nl4 = reinterpret_cast<const float4 *>(mt.neg_lse2 + c * 32);
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 nl = nl4[e >> 2];
+                    float p0 = exp2f(fmaf(__uint_as_float(r[e]), sl2, nl.x));
+                    float p1 = exp2f(fmaf(__uint_as_float(r[e + 1]), sl2, nl.y));
+                    float p2 = exp2f(fmaf(__uint_as_float(r[e + 2]), sl2, nl.z));
+                    float p3 = exp2f(fmaf(__uint_as_float(r[e + 3]), sl2, nl.w));
+                    if (masked) {
+                        p0 = ((mk >> e) & 1u) ? p0 : 0.f;
+                        p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
+                        p2 = ((mk >> (e + 2)) & 1u) ? p2 : 0.f;
+                        p3 = ((mk >> (e + 3)) & 1u) ? p3 : 0.f;
+                    }
+                    pk[e >> 1] = pack_bf16(p0, p1);
+                    pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+                }
+#pragma unroll
+                for (int e = 0; e < 16; ++e) pr[c * 16 + e] = pk[e];
+                tmem_st16(y_addr + c * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm.a_done[b]);
+            // --- phase B: dS^T
+            ok = mbar_wait(&sm.dp_full[b], (t >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t r[32], pk[16];
+                tmem_ld32(x_addr + c * 32, r);
+                tmem_wait_ld();
+                const float4 *dl4 = reinterpret_cast<const float4 *>(mt.delta + c * 32);
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 dl = dl4[e >> 2];
+                    const uint32_t pa = pr[c * 16 + (e >> 1)], pb = pr[c * 16 + (e >> 1) + 1];
+                    const float d0 = __uint_as_float(pa << 16) * (__uint_as_float(r[e]) - dl.x);
+                    const float d1 = __uint_as_float(pa & 0xffff0000u) * (__uint_as_float(r[e + 1]) - dl.y);
+                    const float d2 = __uint_as_float(pb << 16) * (__uint_as_float(r[e + 2]) - dl.z);
+                    const float d3 = __uint_as_float(pb & 0xffff0000u) * (__uint_as_float(r[e + 3]) - dl.w);
+                    pk[e >> 1] = pack_bf16(d0, d1);
+                    pk[(e >> 1) + 1] = pack_bf16(d2, d3);
+                }
+                tmem_st16(y_addr + 32 + c * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm.b_done[b]);
+        }
+        // --- epilogue: warpgroup 0 writes dK (x scale), warpgroup 1 writes dV
+        if (ok && n_iter > 0) ok = mbar_wait(&sm.acc_full, 0, abort_flag);
+        tc_fence_after();
+        const uint32_t acc_addr = tmem + lane_base + b * 128;
+        void *dst = b == 0 ? p.dk : p.dv;
+        const float mul = b == 0 ? p.scale : 1.0f;
+        const size_t base = ((size_t)(gkey0 + (tid & 127)) * p.h_kv + g) * 128;
+        const bool do_store = ok && kvalid;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            if (n_iter > 0 && ok) {
+                tmem_ld32(acc_addr + c * 32, r);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) r[e] = 0u;
+            }
+            if (do_store) {
+                if (p.accumulate) store_grad_chunk<true>(dst, base + c * 32, r, mul);
+                else store_grad_chunk<false>(dst, base + c * 32, r, mul);
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (tid == 0 && sm.abort_flag) atomicExch(p.status, BA_ETIMEOUT);
+}
+
 }  // namespace
 
 int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
@@ -406,8 +768,10 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
               void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st) {
     static bool attr_set = false;
     const size_t dq_smem = sizeof(DqSmem) + 1024;
+    const size_t kv_smem = sizeof(KvSmem) + 1024;
     if (!attr_set) {
         BA_CUDA_CHECK(cudaFuncSetAttribute(tc_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dq_smem));
+        BA_CUDA_CHECK(cudaFuncSetAttribute(tc_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kv_smem));
         attr_set = true;
     }
     const ba_problem_t &pr = pl->prob;
@@ -451,6 +815,22 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
         int rc = ba_check_launch();
         if (rc != BA_OK) return rc;
     }
-    // dK / dV: plain-FMA kernel until the tensor-core one lands
-    return ba_simt_bwd_dkdv(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, dk, dv, st);
+    // dK / dV
+    const int64_t kmt = (r.parts & BA_PART_MAIN) ? (r.kv_end - r.kv_begin + kTile - 1) / kTile : 0;
+    const int64_t kbt = (r.parts & BA_PART_BRANCH) ? (r.tok_end - r.tok_begin + kTile - 1) / kTile : 0;
+    p.main_key_tiles = (int)kmt;
+    p.total_key_tiles = (int)(kmt + kbt);
+    if (p.total_key_tiles > 0) {
+        CUtensorMap tq_main64, tq_branch64, tgo64;
+        if (!make_tmap_rhd(&tq_main64, qm, qm_rows, pr.h_q, 128, kSub) ||
+            !make_tmap_rhd(&tq_branch64, qb, qb_rows, pr.h_q, 128, kSub) ||
+            !make_tmap_rhd(&tgo64, d_o, all_rows, pr.h_q, 128, kSub))
+            return BA_EINVAL;
+        const int64_t grid = (int64_t)p.total_key_tiles * pr.h_kv;
+        if (grid > INT_MAX) return BA_EUNSUPPORTED;
+        tc_dkdv_kernel<<<(unsigned)grid, kKvThreads, kv_smem, st>>>(tq_main64, tq_branch64, tgo64, tk, tv, p);
+        int rc = ba_check_launch();
+        if (rc != BA_OK) return rc;
+    }
+    return BA_OK;
 }
