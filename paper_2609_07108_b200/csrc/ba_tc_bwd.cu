@@ -411,8 +411,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
 //   P^T = exp2(scale_log2 S^T - lse2[col]),  dS^T = P^T o (dP^T - delta[col])
 //   dV_j += P^T dO,  dK_j += dS^T Q          (P^T, dS^T are TMEM A operands)
 // Two sub-tiles are in flight (sets 0 / 1, one softmax warpgroup each).
-//   TMEM: dK [0,128) dV [128,256); set b: X_b = 256 + 128 b (64 cols: S^T, then
-//   dP^T), Y_b = X_b + 64 (P^T in cols [0,32), dS^T in cols [32,64))
+//   TMEM: dK [0,128) dV [128,256); set b: XS_b = 256 + 128 b (64 cols: S^T, its
+//   first 32 columns then hold P^T), XD_b = XS_b + 64 (dP^T, then dS^T)
 constexpr int kKvThreads = 320;
 constexpr int kSub = 64;           // query rows per sub-tile
 constexpr int kQStages = 4;
@@ -432,7 +432,7 @@ struct KvSmem {
     alignas(16) SubMeta meta[kQStages];
     alignas(8) uint64_t kv_full;
     uint64_t q_full[kQStages], q_empty[kQStages];
-    uint64_t s_full[2], a_done[2], dp_full[2], b_done[2], acc_full;
+    uint64_t sd_full[2], pd_done[2], acc_full;
     uint32_t tmem_base;
     int abort_flag;
     int qend_max, bq0_min, bq1_max;
@@ -459,12 +459,10 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
 
     if (tid == 0) {
         mbar_init(&sm.kv_full, 1);
-        for (int s = 0; s < kQStages; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
+        for (int s = 0; s < kQStages; ++s) { mbar_init(&sm.q_full[s], 2); mbar_init(&sm.q_empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&sm.s_full[b], 1);
-            mbar_init(&sm.a_done[b], 128);
-            mbar_init(&sm.dp_full[b], 1);
-            mbar_init(&sm.b_done[b], 128);
+            mbar_init(&sm.sd_full[b], 1);
+            mbar_init(&sm.pd_done[b], 128);
         }
         mbar_init(&sm.acc_full, 1);
         sm.abort_flag = 0;
@@ -532,29 +530,44 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             }
             bool ok = true;
             int issued = 0;
-            for (int t = 0; t < n_iter; ++t) {
-                const int st = t % kQStages;
-                if (t >= kQStages) ok = mbar_wait(&sm.q_empty[st], ((t / kQStages) - 1) & 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
+            // per-row scalars of a sub-tile (2 rows per lane), fetched one
+            // iteration ahead so their latency is off the producer's critical path
+            float nx_lse[2], nx_dl[2];
+            int nx_bs[2];
+            unsigned long long nx_mk[2];
+            auto fetch = [&](int t) {
                 const int h = g * p.group + t / n_sub;
                 const int s = t % n_sub;
                 const bool seg_main = s < n_sub_main;
                 const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
                 const int64_t rend = seg_main ? m1 : b1;
                 const int64_t grow0 = seg_main ? r0 : n + r0;
-                SubMeta &mt = sm.meta[st];
-                for (int c = lane; c < kSub; c += 32) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int c = lane + 32 * u;
                     const bool live = r0 + c < rend;
-                    mt.neg_lse2[c] = live ? -p.lse[(grow0 + c) * p.h_q + h] * kLog2e : -INFINITY;
-                    mt.delta[c] = live ? p.delta[(grow0 + c) * p.h_q + h] : 0.f;
-                    if (!main_keys) {
-                        mt.bstart[c] = live ? p.meta.br_start[r0 + c] : 0;
-                        mt.mask[c] = live ? p.meta.br_mask[r0 + c] : 0ull;
+                    nx_lse[u] = live ? -p.lse[(grow0 + c) * p.h_q + h] * kLog2e : -INFINITY;
+                    nx_dl[u] = live ? p.delta[(grow0 + c) * p.h_q + h] : 0.f;
+                    nx_bs[u] = 0;
+                    nx_mk[u] = 0ull;
+                    if (!main_keys && live) {
+                        nx_bs[u] = p.meta.br_start[r0 + c];
+                        nx_mk[u] = p.meta.br_mask[r0 + c];
                     }
                 }
-                __syncwarp();
+            };
+            fetch(0);
+            for (int t = 0; t < n_iter; ++t) {
+                const int st = t % kQStages;
+                if (t >= kQStages) ok = mbar_wait(&sm.q_empty[st], ((t / kQStages) - 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
                 if (lane == 0) {
+                    const int h = g * p.group + t / n_sub;
+                    const int s = t % n_sub;
+                    const bool seg_main = s < n_sub_main;
+                    const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
+                    const int64_t grow0 = seg_main ? r0 : n + r0;
                     const CUtensorMap *tq = seg_main ? &tm_q_main : &tm_q_branch;
                     mbar_expect_tx(&sm.q_full[st], 2 * kSubBytes);
                     for (int half = 0; half < 2; ++half) {
@@ -563,6 +576,20 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
                                     &sm.q_full[st]);
                     }
                 }
+                SubMeta &mt = sm.meta[st];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int c = lane + 32 * u;
+                    mt.neg_lse2[c] = nx_lse[u];
+                    mt.delta[c] = nx_dl[u];
+                    if (!main_keys) {
+                        mt.bstart[c] = nx_bs[u];
+                        mt.mask[c] = nx_mk[u];
+                    }
+                }
+                if (t + 1 < n_iter) fetch(t + 1);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.q_full[st]);  // second arrival: the scalars are in place
                 issued = t + 1;
             }
             if (!ok && lane == 0) {
@@ -598,38 +625,28 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
                 ok = mbar_wait(&sm.q_full[b], 0, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_t(tmem + 256 + b * 128, k_addr, smem_u32(sm.qs[b]));
-                tc_commit(&sm.s_full[b]);
+                issue_t(tmem + 256 + b * 128, k_addr, smem_u32(sm.qs[b]));                    // S^T = K Q^T
+                issue_t(tmem + 256 + b * 128 + 64, v_addr, smem_u32(sm.qs[b]) + kSubBytes);   // dP^T = V dO^T
+                tc_commit(&sm.sd_full[b]);
             }
-            for (int t0 = 0; t0 < n_iter && ok; t0 += 2) {
-                for (int b = 0; b < 2 && ok; ++b) {
-                    const int t = t0 + b;
-                    if (t >= n_iter) break;
-                    const uint32_t stage_addr = smem_u32(sm.qs[t % kQStages]);
-                    ok = mbar_wait(&sm.a_done[b], (t >> 1) & 1, abort_flag);
+            for (int t = 0; t < n_iter && ok; ++t) {
+                const int b = t & 1;
+                const uint32_t stage_addr = smem_u32(sm.qs[t % kQStages]);
+                ok = mbar_wait(&sm.pd_done[b], (t >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                issue_acc(tmem + 128, tmem + 256 + b * 128, stage_addr + kSubBytes, t > 0);   // dV += P^T dO
+                issue_acc(tmem + 0, tmem + 256 + b * 128 + 64, stage_addr, t > 0);             // dK += dS^T Q
+                tc_commit(&sm.q_empty[t % kQStages]);
+                const int t2 = t + 2;
+                if (t2 < n_iter) {
+                    const uint32_t next_addr = smem_u32(sm.qs[t2 % kQStages]);
+                    ok = mbar_wait(&sm.q_full[t2 % kQStages], (t2 / kQStages) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_t(tmem + 256 + b * 128, v_addr, stage_addr + kSubBytes);     // dP^T = V dO^T
-                    tc_commit(&sm.dp_full[b]);
-                    issue_acc(tmem + 128, tmem + 256 + b * 128 + 64, stage_addr + kSubBytes, t > 0);  // dV += P^T dO
-                }
-                for (int b = 0; b < 2 && ok; ++b) {
-                    const int t = t0 + b;
-                    if (t >= n_iter) break;
-                    const uint32_t stage_addr = smem_u32(sm.qs[t % kQStages]);
-                    ok = mbar_wait(&sm.b_done[b], (t >> 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_acc(tmem + 0, tmem + 256 + b * 128 + 96, stage_addr, t > 0);                // dK += dS^T Q
-                    tc_commit(&sm.q_empty[t % kQStages]);
-                    const int t2 = t + 2;
-                    if (t2 < n_iter) {
-                        ok = mbar_wait(&sm.q_full[t2 % kQStages], (t2 / kQStages) & 1, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_t(tmem + 256 + b * 128, k_addr, smem_u32(sm.qs[t2 % kQStages]));
-                        tc_commit(&sm.s_full[b]);
-                    }
+                    issue_t(tmem + 256 + b * 128, k_addr, next_addr);
+                    issue_t(tmem + 256 + b * 128 + 64, v_addr, next_addr + kSubBytes);
+                    tc_commit(&sm.sd_full[b]);
                 }
             }
             if (ok) tc_commit(&sm.acc_full);
@@ -638,8 +655,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
         // ================================================= P^T / dS^T warps + epilogue
         const int b = warp >> 2;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t x_addr = tmem + lane_base + 256 + b * 128;
-        const uint32_t y_addr = x_addr + 64;
+        const uint32_t xs_addr = tmem + lane_base + 256 + b * 128;
+        const uint32_t xd_addr = xs_addr + 64;
         const float sl2 = p.scale_log2;
         bool ok = true;
         for (int t = b; t < n_iter; t += 2) {
@@ -649,11 +666,10 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
             const int64_t rend = seg_main ? m1 : b1;
             const SubMeta &mt = sm.meta[st];
-            ok = mbar_wait(&sm.s_full[b], (t >> 1) & 1, abort_flag);
-            ok = ok && mbar_wait(&sm.q_full[st], (t / kQStages) & 1, abort_flag);  // metadata of the stage
+            // --- which of the 64 query rows (columns) see my key (needs only the
+            // stage's scalars, so it runs while the MMAs are still in flight)
+            ok = mbar_wait(&sm.q_full[st], (t / kQStages) & 1, abort_flag);
             if (!ok) break;
-            tc_fence_after();
-            // --- which of the 64 query rows (columns) see my key
             uint64_t vis = 0ull;
             if (kvalid) {
                 if (main_keys) {
@@ -671,22 +687,26 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
                 }
             }
             const bool masked = !__all_sync(0xffffffffu, vis == ~0ull);
-            // --- phase A: P^T
-            uint32_t pr[32];
+            ok = mbar_wait(&sm.sd_full[b], (t >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            // --- P^T = exp2(scale_log2 S^T - lse2[col]), dS^T = P^T o (dP^T - delta[col])
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
-                uint32_t r[32], pk[16];
-                tmem_ld32(x_addr + c * 32, r);
+                uint32_t rs[32], rd[32], pk[16], dk16[16];
+                tmem_ld32(xs_addr + c * 32, rs);
+                tmem_ld32(xd_addr + c * 32, rd);
                 tmem_wait_ld();
                 const uint32_t mk = masked ? (uint32_t)(vis >> (c * 32)) : 0xffffffffu;
                 const float4 *nl4 = reinterpret_cast<const float4 *>(mt.neg_lse2 + c * 32);
+                const float4 *dl4 = reinterpret_cast<const float4 *>(mt.delta + c * 32);
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                    const float4 nl = nl4[e >> 2];
-                    float p0 = exp2f(fmaf(__uint_as_float(r[e]), sl2, nl.x));
-                    float p1 = exp2f(fmaf(__uint_as_float(r[e + 1]), sl2, nl.y));
-                    float p2 = exp2f(fmaf(__uint_as_float(r[e + 2]), sl2, nl.z));
-                    float p3 = exp2f(fmaf(__uint_as_float(r[e + 3]), sl2, nl.w));
+                    const float4 nl = nl4[e >> 2], dl = dl4[e >> 2];
+                    float p0 = exp2f(fmaf(__uint_as_float(rs[e]), sl2, nl.x));
+                    float p1 = exp2f(fmaf(__uint_as_float(rs[e + 1]), sl2, nl.y));
+                    float p2 = exp2f(fmaf(__uint_as_float(rs[e + 2]), sl2, nl.z));
+                    float p3 = exp2f(fmaf(__uint_as_float(rs[e + 3]), sl2, nl.w));
                     if (masked) {
                         p0 = ((mk >> e) & 1u) ? p0 : 0.f;
                         p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
@@ -695,40 +715,15 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
                     }
                     pk[e >> 1] = pack_bf16(p0, p1);
                     pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+                    dk16[e >> 1] = pack_bf16(p0 * (__uint_as_float(rd[e]) - dl.x), p1 * (__uint_as_float(rd[e + 1]) - dl.y));
+                    dk16[(e >> 1) + 1] = pack_bf16(p2 * (__uint_as_float(rd[e + 2]) - dl.z), p3 * (__uint_as_float(rd[e + 3]) - dl.w));
                 }
-#pragma unroll
-                for (int e = 0; e < 16; ++e) pr[c * 16 + e] = pk[e];
-                tmem_st16(y_addr + c * 16, pk);
+                tmem_st16(xs_addr + c * 16, pk);
+                tmem_st16(xd_addr + c * 16, dk16);
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&sm.a_done[b]);
-            // --- phase B: dS^T
-            ok = mbar_wait(&sm.dp_full[b], (t >> 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t r[32], pk[16];
-                tmem_ld32(x_addr + c * 32, r);
-                tmem_wait_ld();
-                const float4 *dl4 = reinterpret_cast<const float4 *>(mt.delta + c * 32);
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const float4 dl = dl4[e >> 2];
-                    const uint32_t pa = pr[c * 16 + (e >> 1)], pb = pr[c * 16 + (e >> 1) + 1];
-                    const float d0 = __uint_as_float(pa << 16) * (__uint_as_float(r[e]) - dl.x);
-                    const float d1 = __uint_as_float(pa & 0xffff0000u) * (__uint_as_float(r[e + 1]) - dl.y);
-                    const float d2 = __uint_as_float(pb << 16) * (__uint_as_float(r[e + 2]) - dl.z);
-                    const float d3 = __uint_as_float(pb & 0xffff0000u) * (__uint_as_float(r[e + 3]) - dl.w);
-                    pk[e >> 1] = pack_bf16(d0, d1);
-                    pk[(e >> 1) + 1] = pack_bf16(d2, d3);
-                }
-                tmem_st16(y_addr + 32 + c * 16, pk);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(&sm.b_done[b]);
+            mbar_arrive(&sm.pd_done[b]);
         }
         // --- epilogue: warpgroup 0 writes dK (x scale), warpgroup 1 writes dV
         if (ok && n_iter > 0) ok = mbar_wait(&sm.acc_full, 0, abort_flag);
