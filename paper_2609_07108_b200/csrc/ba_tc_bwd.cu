@@ -92,6 +92,36 @@ __device__ __forceinline__ void store_grad_chunk(void *dst, size_t elem_off, con
     }
 }
 
+// P = 2^(s * sl2 + neg_lse2) for one 32-column chunk, as 16 packed bf16 pairs
+template <bool MASKED>
+__device__ __forceinline__ void chunk_p(const uint32_t (&r)[32], uint32_t mk, float sl2, float neg_lse2,
+                                        uint32_t *pr) {
+    const float2 s2 = make_float2(sl2, sl2), n2 = make_float2(neg_lse2, neg_lse2);
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        const float2 x = ffma2(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), s2, n2);
+        float p0 = ex2(x.x), p1 = ex2(x.y);
+        if (MASKED) {
+            p0 = ((mk >> e) & 1u) ? p0 : 0.f;
+            p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
+        }
+        pr[e >> 1] = pack_bf16(p0, p1);
+    }
+}
+
+// dS = P o (dP - delta) for one 32-column chunk (P given as packed bf16 pairs)
+__device__ __forceinline__ void chunk_ds(const uint32_t (&r)[32], const uint32_t *pr, float dlt,
+                                         uint32_t (&pk)[16]) {
+    const float2 nd = make_float2(-dlt, -dlt);
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        const uint32_t pp = pr[e >> 1];
+        const float2 pf = make_float2(__uint_as_float(pp << 16), __uint_as_float(pp & 0xffff0000u));
+        const float2 d = fmul2(pf, fadd2(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), nd));
+        pk[e >> 1] = pack_bf16(d.x, d.y);
+    }
+}
+
 __global__ void __launch_bounds__(kDqThreads, 1)
 tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constant__ CUtensorMap tm_q_branch,
              const __grid_constant__ CUtensorMap tm_go, const __grid_constant__ CUtensorMap tm_k,
@@ -329,23 +359,28 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
             ok = mbar_wait(&sm.s_full[i], j & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            uint32_t pr[64];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(r_addr + c * 32, r);
+            const uint32_t mk0 = (uint32_t)vis[0], mk1 = (uint32_t)(vis[0] >> 32);
+            const uint32_t mk2 = (uint32_t)vis[1], mk3 = (uint32_t)(vis[1] >> 32);
+            uint32_t pr[64], ra[32], rb[32];
+            tmem_ld32(r_addr, ra);
+            tmem_ld32(r_addr + 32, rb);
+            tmem_wait_ld();
+            if (masked) {
+                chunk_p<true>(ra, mk0, sl2, neg_lse2, &pr[0]);
+                tmem_ld32(r_addr + 64, ra);
+                chunk_p<true>(rb, mk1, sl2, neg_lse2, &pr[16]);
+                tmem_ld32(r_addr + 96, rb);
                 tmem_wait_ld();
-                const uint32_t mk = masked ? (uint32_t)(vis[c >> 1] >> ((c & 1) * 32)) : 0xffffffffu;
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float p0 = exp2f(fmaf(__uint_as_float(r[e]), sl2, neg_lse2));
-                    float p1 = exp2f(fmaf(__uint_as_float(r[e + 1]), sl2, neg_lse2));
-                    if (masked) {
-                        p0 = ((mk >> e) & 1u) ? p0 : 0.f;
-                        p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
-                    }
-                    pr[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
-                }
+                chunk_p<true>(ra, mk2, sl2, neg_lse2, &pr[32]);
+                chunk_p<true>(rb, mk3, sl2, neg_lse2, &pr[48]);
+            } else {
+                chunk_p<false>(ra, 0u, sl2, neg_lse2, &pr[0]);
+                tmem_ld32(r_addr + 64, ra);
+                chunk_p<false>(rb, 0u, sl2, neg_lse2, &pr[16]);
+                tmem_ld32(r_addr + 96, rb);
+                tmem_wait_ld();
+                chunk_p<false>(ra, 0u, sl2, neg_lse2, &pr[32]);
+                chunk_p<false>(rb, 0u, sl2, neg_lse2, &pr[48]);
             }
             tc_fence_before();
             mbar_arrive(&sm.a_done[i]);
@@ -353,18 +388,22 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
             ok = mbar_wait(&sm.dp_full[i], j & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32], pk[16];
-                tmem_ld32(r_addr + c * 32, r);
+            {
+                uint32_t pk[16];
+                tmem_ld32(r_addr, ra);
+                tmem_ld32(r_addr + 32, rb);
                 tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const uint32_t pp = pr[c * 16 + (e >> 1)];
-                    const float p0 = __uint_as_float(pp << 16), p1 = __uint_as_float(pp & 0xffff0000u);
-                    pk[e >> 1] = pack_bf16(p0 * (__uint_as_float(r[e]) - dlt), p1 * (__uint_as_float(r[e + 1]) - dlt));
-                }
-                tmem_st16(r_addr + c * 16, pk);
+                chunk_ds(ra, &pr[0], dlt, pk);
+                tmem_st16(r_addr, pk);
+                tmem_ld32(r_addr + 64, ra);
+                chunk_ds(rb, &pr[16], dlt, pk);
+                tmem_st16(r_addr + 16, pk);
+                tmem_ld32(r_addr + 96, rb);
+                tmem_wait_ld();
+                chunk_ds(ra, &pr[32], dlt, pk);
+                tmem_st16(r_addr + 32, pk);
+                chunk_ds(rb, &pr[48], dlt, pk);
+                tmem_st16(r_addr + 48, pk);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -437,6 +476,40 @@ struct KvSmem {
     int abort_flag;
     int qend_max, bq0_min, bq1_max;
 };
+
+// 16 columns of the transposed tile: P^T and dS^T as 8 packed bf16 pairs each;
+// nl / dl point at the columns' -lse2 and delta in shared memory
+template <bool MASKED>
+__device__ __forceinline__ void quarter_pds(const uint32_t (&rs)[16], const uint32_t (&rd)[16], uint32_t mk,
+                                            float sl2, const float *nl, const float *dl, uint32_t (&pk)[8],
+                                            uint32_t (&dk8)[8]) {
+    const float2 s2 = make_float2(sl2, sl2);
+    const float4 *nl4 = reinterpret_cast<const float4 *>(nl);
+    const float4 *dl4 = reinterpret_cast<const float4 *>(dl);
+#pragma unroll
+    for (int e = 0; e < 16; e += 4) {
+        const float4 nv = nl4[e >> 2], dv = dl4[e >> 2];
+        const float2 x0 = ffma2(make_float2(__uint_as_float(rs[e]), __uint_as_float(rs[e + 1])), s2,
+                                make_float2(nv.x, nv.y));
+        const float2 x1 = ffma2(make_float2(__uint_as_float(rs[e + 2]), __uint_as_float(rs[e + 3])), s2,
+                                make_float2(nv.z, nv.w));
+        float2 p0 = make_float2(ex2(x0.x), ex2(x0.y)), p1 = make_float2(ex2(x1.x), ex2(x1.y));
+        if (MASKED) {
+            p0.x = ((mk >> e) & 1u) ? p0.x : 0.f;
+            p0.y = ((mk >> (e + 1)) & 1u) ? p0.y : 0.f;
+            p1.x = ((mk >> (e + 2)) & 1u) ? p1.x : 0.f;
+            p1.y = ((mk >> (e + 3)) & 1u) ? p1.y : 0.f;
+        }
+        const float2 d0 = fmul2(p0, fadd2(make_float2(__uint_as_float(rd[e]), __uint_as_float(rd[e + 1])),
+                                          make_float2(-dv.x, -dv.y)));
+        const float2 d1 = fmul2(p1, fadd2(make_float2(__uint_as_float(rd[e + 2]), __uint_as_float(rd[e + 3])),
+                                          make_float2(-dv.z, -dv.w)));
+        pk[e >> 1] = pack_bf16(p0.x, p0.y);
+        pk[(e >> 1) + 1] = pack_bf16(p1.x, p1.y);
+        dk8[e >> 1] = pack_bf16(d0.x, d0.y);
+        dk8[(e >> 1) + 1] = pack_bf16(d1.x, d1.y);
+    }
+}
 
 __global__ void __launch_bounds__(kKvThreads, 1)
 tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constant__ CUtensorMap tm_q_branch,
@@ -690,36 +763,40 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             ok = mbar_wait(&sm.sd_full[b], (t >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            // --- P^T = exp2(scale_log2 S^T - lse2[col]), dS^T = P^T o (dP^T - delta[col])
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t rs[32], rd[32], pk[16], dk16[16];
-                tmem_ld32(xs_addr + c * 32, rs);
-                tmem_ld32(xd_addr + c * 32, rd);
+            // --- P^T = exp2(scale_log2 S^T - lse2[col]), dS^T = P^T o (dP^T - delta[col]),
+            // 16 columns at a time, the next pair of loads in flight behind the math
+            {
+                uint32_t sa[16], da[16], sb[16], db[16], pk[8], dk8[8];
+                tmem_ld16(xs_addr, sa);
+                tmem_ld16(xd_addr, da);
+                tmem_ld16(xs_addr + 16, sb);
+                tmem_ld16(xd_addr + 16, db);
                 tmem_wait_ld();
-                const uint32_t mk = masked ? (uint32_t)(vis >> (c * 32)) : 0xffffffffu;
-                const float4 *nl4 = reinterpret_cast<const float4 *>(mt.neg_lse2 + c * 32);
-                const float4 *dl4 = reinterpret_cast<const float4 *>(mt.delta + c * 32);
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const float4 nl = nl4[e >> 2], dl = dl4[e >> 2];
-                    float p0 = exp2f(fmaf(__uint_as_float(rs[e]), sl2, nl.x));
-                    float p1 = exp2f(fmaf(__uint_as_float(rs[e + 1]), sl2, nl.y));
-                    float p2 = exp2f(fmaf(__uint_as_float(rs[e + 2]), sl2, nl.z));
-                    float p3 = exp2f(fmaf(__uint_as_float(rs[e + 3]), sl2, nl.w));
-                    if (masked) {
-                        p0 = ((mk >> e) & 1u) ? p0 : 0.f;
-                        p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
-                        p2 = ((mk >> (e + 2)) & 1u) ? p2 : 0.f;
-                        p3 = ((mk >> (e + 3)) & 1u) ? p3 : 0.f;
-                    }
-                    pk[e >> 1] = pack_bf16(p0, p1);
-                    pk[(e >> 1) + 1] = pack_bf16(p2, p3);
-                    dk16[e >> 1] = pack_bf16(p0 * (__uint_as_float(rd[e]) - dl.x), p1 * (__uint_as_float(rd[e + 1]) - dl.y));
-                    dk16[(e >> 1) + 1] = pack_bf16(p2 * (__uint_as_float(rd[e + 2]) - dl.z), p3 * (__uint_as_float(rd[e + 3]) - dl.w));
+                if (masked) {
+                    quarter_pds<true>(sa, da, (uint32_t)vis & 0xffffu, sl2, mt.neg_lse2, mt.delta, pk, dk8);
+                    tmem_st8(xs_addr, pk); tmem_st8(xd_addr, dk8);
+                    tmem_ld16(xs_addr + 32, sa); tmem_ld16(xd_addr + 32, da);
+                    quarter_pds<true>(sb, db, (uint32_t)(vis >> 16) & 0xffffu, sl2, mt.neg_lse2 + 16, mt.delta + 16, pk, dk8);
+                    tmem_st8(xs_addr + 8, pk); tmem_st8(xd_addr + 8, dk8);
+                    tmem_ld16(xs_addr + 48, sb); tmem_ld16(xd_addr + 48, db);
+                    tmem_wait_ld();
+                    quarter_pds<true>(sa, da, (uint32_t)(vis >> 32) & 0xffffu, sl2, mt.neg_lse2 + 32, mt.delta + 32, pk, dk8);
+                    tmem_st8(xs_addr + 16, pk); tmem_st8(xd_addr + 16, dk8);
+                    quarter_pds<true>(sb, db, (uint32_t)(vis >> 48) & 0xffffu, sl2, mt.neg_lse2 + 48, mt.delta + 48, pk, dk8);
+                    tmem_st8(xs_addr + 24, pk); tmem_st8(xd_addr + 24, dk8);
+                } else {
+                    quarter_pds<false>(sa, da, 0u, sl2, mt.neg_lse2, mt.delta, pk, dk8);
+                    tmem_st8(xs_addr, pk); tmem_st8(xd_addr, dk8);
+                    tmem_ld16(xs_addr + 32, sa); tmem_ld16(xd_addr + 32, da);
+                    quarter_pds<false>(sb, db, 0u, sl2, mt.neg_lse2 + 16, mt.delta + 16, pk, dk8);
+                    tmem_st8(xs_addr + 8, pk); tmem_st8(xd_addr + 8, dk8);
+                    tmem_ld16(xs_addr + 48, sb); tmem_ld16(xd_addr + 48, db);
+                    tmem_wait_ld();
+                    quarter_pds<false>(sa, da, 0u, sl2, mt.neg_lse2 + 32, mt.delta + 32, pk, dk8);
+                    tmem_st8(xs_addr + 16, pk); tmem_st8(xd_addr + 16, dk8);
+                    quarter_pds<false>(sb, db, 0u, sl2, mt.neg_lse2 + 48, mt.delta + 48, pk, dk8);
+                    tmem_st8(xs_addr + 24, pk); tmem_st8(xd_addr + 24, dk8);
                 }
-                tmem_st16(xs_addr + c * 16, pk);
-                tmem_st16(xd_addr + c * 16, dk16);
             }
             tmem_wait_st();
             tc_fence_before();

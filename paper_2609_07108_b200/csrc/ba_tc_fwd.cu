@@ -88,6 +88,44 @@ __device__ __forceinline__ void store_row_chunk(void *o, size_t elem_off, const 
     }
 }
 
+// max over one 32-column chunk of scores (masked columns count as -inf)
+template <bool MASKED>
+__device__ __forceinline__ float chunk_max(const uint32_t (&r)[32], uint32_t mk, float m) {
+    float m0 = m, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        float a = __uint_as_float(r[e]), b = __uint_as_float(r[e + 1]);
+        float c = __uint_as_float(r[e + 2]), d = __uint_as_float(r[e + 3]);
+        if (MASKED) {
+            a = ((mk >> e) & 1u) ? a : -INFINITY;
+            b = ((mk >> (e + 1)) & 1u) ? b : -INFINITY;
+            c = ((mk >> (e + 2)) & 1u) ? c : -INFINITY;
+            d = ((mk >> (e + 3)) & 1u) ? d : -INFINITY;
+        }
+        m0 = fmaxf(m0, a); m1 = fmaxf(m1, b); m2 = fmaxf(m2, c); m3 = fmaxf(m3, d);
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// p = 2^(s * sl2 + neg_ms) for one 32-column chunk -> 16 packed bf16 pairs; the
+// row sum is kept as two partial sums (packed fp32 add)
+template <bool MASKED>
+__device__ __forceinline__ void chunk_exp(const uint32_t (&r)[32], uint32_t mk, float sl2, float neg_ms,
+                                          float2 &lsum, uint32_t (&pk)[16]) {
+    const float2 s2 = make_float2(sl2, sl2), n2 = make_float2(neg_ms, neg_ms);
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        const float2 x = ffma2(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), s2, n2);
+        float2 pp = make_float2(ex2(x.x), ex2(x.y));
+        if (MASKED) {
+            pp.x = ((mk >> e) & 1u) ? pp.x : 0.f;
+            pp.y = ((mk >> (e + 1)) & 1u) ? pp.y : 0.f;
+        }
+        lsum = fadd2(lsum, pp);
+        pk[e >> 1] = pack_bf16(pp.x, pp.y);
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constant__ CUtensorMap tm_q_branch,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -310,29 +348,37 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                     else { vis[0] = 0ull; vis[1] = 0ull; }
                 }
             }
-            // --- pass 1: row maximum
-            float m_tile = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(s_addr + c * 32, r);
+            const uint32_t mk0 = (uint32_t)vis[0], mk1 = (uint32_t)(vis[0] >> 32);
+            const uint32_t mk2 = (uint32_t)vis[1], mk3 = (uint32_t)(vis[1] >> 32);
+            // --- pass 1: row maximum (chunks 2, 3, then 0, 1, which stay in registers)
+            uint32_t ra[32], rb[32];
+            float m_tile;
+            tmem_ld32(s_addr + 64, ra);
+            tmem_ld32(s_addr + 96, rb);
+            tmem_wait_ld();
+            if (masked) {
+                m_tile = chunk_max<true>(ra, mk2, -INFINITY);
+                tmem_ld32(s_addr, ra);
+                m_tile = chunk_max<true>(rb, mk3, m_tile);
+                tmem_ld32(s_addr + 32, rb);
                 tmem_wait_ld();
-                if (masked) {
-                    const uint32_t mk = (uint32_t)(vis[c >> 1] >> ((c & 1) * 32));
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        m_tile = fmaxf(m_tile, ((mk >> e) & 1u) ? __uint_as_float(r[e]) : -INFINITY);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) m_tile = fmaxf(m_tile, __uint_as_float(r[e]));
-                }
+                m_tile = chunk_max<true>(ra, mk0, m_tile);
+                m_tile = chunk_max<true>(rb, mk1, m_tile);
+            } else {
+                m_tile = chunk_max<false>(ra, 0u, -INFINITY);
+                tmem_ld32(s_addr, ra);
+                m_tile = chunk_max<false>(rb, 0u, m_tile);
+                tmem_ld32(s_addr + 32, rb);
+                tmem_wait_ld();
+                m_tile = chunk_max<false>(ra, 0u, m_tile);
+                m_tile = chunk_max<false>(rb, 0u, m_tile);
             }
             // --- running maximum; O and l are rescaled only when it grew a lot
             const float m_new = fmaxf(m_run, m_tile);
             float alpha = 1.0f;
             const bool grow = m_new > m_run && (m_run == -INFINITY || (m_new - m_run) * sl2 > kRescaleThreshold);
             if (grow) {
-                alpha = exp2f((m_run - m_new) * sl2);  // m_run = -inf gives 0
+                alpha = ex2((m_run - m_new) * sl2);  // m_run = -inf gives 0
                 l_run *= alpha;
                 m_run = m_new;
             }
@@ -349,26 +395,34 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
             }
             const float neg_ms = m_run == -INFINITY ? 0.f : -m_run * sl2;
             // --- pass 2: P = exp2(s * scale_log2 - m), bf16, over the first 64 score columns
-            float l_add = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32], pk[16];
-                tmem_ld32(s_addr + c * 32, r);
+            float2 l2 = make_float2(0.f, 0.f);
+            uint32_t pk[16];
+            if (masked) {
+                chunk_exp<true>(ra, mk0, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr, pk);
+                tmem_ld32(s_addr + 64, ra);
+                chunk_exp<true>(rb, mk1, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr + 16, pk);
+                tmem_ld32(s_addr + 96, rb);
                 tmem_wait_ld();
-                const uint32_t mk = masked ? (uint32_t)(vis[c >> 1] >> ((c & 1) * 32)) : 0xffffffffu;
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float p0 = exp2f(fmaf(__uint_as_float(r[e]), sl2, neg_ms));
-                    float p1 = exp2f(fmaf(__uint_as_float(r[e + 1]), sl2, neg_ms));
-                    if (masked) {
-                        p0 = ((mk >> e) & 1u) ? p0 : 0.f;
-                        p1 = ((mk >> (e + 1)) & 1u) ? p1 : 0.f;
-                    }
-                    l_add += p0 + p1;
-                    pk[e >> 1] = pack_bf16(p0, p1);
-                }
-                tmem_st16(s_addr + c * 16, pk);
+                chunk_exp<true>(ra, mk2, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr + 32, pk);
+                chunk_exp<true>(rb, mk3, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr + 48, pk);
+            } else {
+                chunk_exp<false>(ra, 0u, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr, pk);
+                tmem_ld32(s_addr + 64, ra);
+                chunk_exp<false>(rb, 0u, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr + 16, pk);
+                tmem_ld32(s_addr + 96, rb);
+                tmem_wait_ld();
+                chunk_exp<false>(ra, 0u, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr + 32, pk);
+                chunk_exp<false>(rb, 0u, sl2, neg_ms, l2, pk);
+                tmem_st16(s_addr + 48, pk);
             }
+            const float l_add = l2.x + l2.y;
             l_run += l_add;
             tmem_wait_st();
             tc_fence_before();
