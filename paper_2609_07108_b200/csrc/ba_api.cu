@@ -39,8 +39,8 @@ int make_range(const ba_plan *pl, int64_t qm_begin, int64_t qm_end, int64_t br_b
 
 extern "C" size_t ba_workspace_bytes(const ba_plan_t *plan, int op) {
     if (!plan) return 0;
-    if (op == BA_OP_BWD)  // delta = rowsum(dO * O), fp32 [N + M, h_q]
-        return align256((size_t)(plan->prob.n_main + plan->prob.n_branch) * plan->prob.h_q * sizeof(float));
+    if (op == BA_OP_BWD)  // delta and -LSE*log2(e), fp32, head-major [h_q, row_pitch] each
+        return align256((size_t)2 * plan->row_pitch * plan->prob.h_q * sizeof(float));
     return 0;
 }
 
@@ -104,11 +104,13 @@ extern "C" int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const 
     if (!workspace || ws_bytes < need || ((uintptr_t)workspace & 255)) return BA_EWORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     float *delta = (float *)workspace;
+    float *nlse2 = delta + (size_t)plan->row_pitch * plan->prob.h_q;
+    const int64_t rp = plan->row_pitch;
     const int64_t n = plan->prob.n_main;
     const int hq = plan->prob.h_q, d = plan->prob.head_dim, dt = plan->prob.dtype;
-    if (has_main_q && (rc = ba_delta(O, dO, delta, r.qm_begin, r.qm_end, hq, d, dt, st)) != BA_OK) return rc;
+    if (has_main_q && (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, r.qm_begin, r.qm_end, hq, d, dt, st)) != BA_OK) return rc;
     if (has_branch_q &&
-        (rc = ba_delta(O, dO, delta, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
+        (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
         return rc;
     const void *qm = has_main_q ? q_main : nullptr;
     if (plan->impl == BA_IMPL_TC)

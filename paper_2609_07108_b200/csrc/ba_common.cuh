@@ -27,6 +27,7 @@ struct ba_plan {
     float scale;
     int impl;                     // BA_IMPL_SIMT or BA_IMPL_TC (resolved)
     int64_t pairs;
+    int64_t row_pitch;            // rows per head of the head-major backward scratch (>= N + M + 128)
     int32_t *host_offsets;        // host copy of branch_offsets (NULL when uniform_len > 0)
     int32_t *dev_status;          // one int32 in plan_mem: device-side status word
 };
@@ -81,5 +82,9 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
               void *dv, cudaStream_t st);
 bool ba_tc_supported(const ba_problem_t *p);
 // Elementwise (ba_elementwise.cu)
-int ba_delta(const void *o, const void *d_o, float *delta, int64_t row_begin, int64_t row_end,
-             int h_q, int d, int dtype, cudaStream_t st);
+// Backward preprocess into head-major scratch [h_q, row_pitch]:
+//   delta_t[h, r] = <dO[r, h], O[r, h]>,  nlse2_t[h, r] = -LSE[r, h] * log2(e)
+int ba_delta(const void *o, const void *d_o, const float *lse, float *delta_t, float *nlse2_t,
+             int64_t row_pitch, int64_t row_begin, int64_t row_end, int h_q, int d, int dtype,
+             cudaStream_t st);
+static inline int64_t ba_row_pitch(int64_t rows) { return (rows + 128 + 63) / 64 * 64; }

@@ -94,11 +94,13 @@ int launch_merge(int lpi, int64_t items, const float *oa, const float *la, const
     return ba_check_launch();
 }
 
-// delta[r, h] = sum_d dO[r, h, d] * O[r, h, d]; one 16-byte chunk per lane.
+// delta_t[h, r] = sum_d dO[r, h, d] * O[r, h, d] and nlse2_t[h, r] = -LSE[r, h] log2(e),
+// both head-major with `pitch` rows per head; one 16-byte chunk per lane.
 template <typename T, int LPI>
 __global__ void __launch_bounds__(kThreads)
 delta_kernel(int64_t items, const uint4 *__restrict__ o, const uint4 *__restrict__ d_o,
-             float *__restrict__ delta) {
+             const float *__restrict__ lse, float *__restrict__ delta_t, float *__restrict__ nlse2_t,
+             int64_t row_begin, int h_q, int64_t pitch) {
     constexpr int IPW = 32 / LPI;
     const int lane = threadIdx.x & 31;
     const int sub = lane % LPI;
@@ -126,7 +128,12 @@ delta_kernel(int64_t items, const uint4 *__restrict__ o, const uint4 *__restrict
         }
 #pragma unroll
         for (int off = LPI / 2; off; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (i < items && sub == 0) delta[i] = acc;
+        if (i < items && sub == 0) {
+            const int64_t r = row_begin + i / h_q;
+            const int h = (int)(i % h_q);
+            delta_t[h * pitch + r] = acc;
+            nlse2_t[h * pitch + r] = -lse[r * h_q + h] * 1.4426950408889634f;
+        }
     }
 }
 
@@ -169,26 +176,25 @@ extern "C" int lse_merge(int64_t rows_heads, int d, const float *O_a, const floa
     return launch_merge<false>(d / 4, rows_heads, O_a, LSE_a, O_b, LSE_b, O_out, LSE_out, st);
 }
 
-int ba_delta(const void *o, const void *d_o, float *delta, int64_t row_begin, int64_t row_end,
-             int h_q, int d, int dtype, cudaStream_t st) {
+int ba_delta(const void *o, const void *d_o, const float *lse, float *delta_t, float *nlse2_t,
+             int64_t row_pitch, int64_t row_begin, int64_t row_end, int h_q, int d, int dtype,
+             cudaStream_t st) {
     const int64_t items = (row_end - row_begin) * h_q;
     if (items <= 0) return BA_OK;
     const size_t esz = dtype == BA_FP32 ? 4 : 2;
-    const char *op = (const char *)o + (size_t)row_begin * h_q * d * esz;
-    const char *gp = (const char *)d_o + (size_t)row_begin * h_q * d * esz;
-    float *dp = delta + row_begin * h_q;
+    const uint4 *op = (const uint4 *)((const char *)o + (size_t)row_begin * h_q * d * esz);
+    const uint4 *gp = (const uint4 *)((const char *)d_o + (size_t)row_begin * h_q * d * esz);
     const int lpi = (int)(d * esz / 16);
     const int grid = stream_grid(items * lpi);
-    if (dtype == BA_FP32 && lpi == 16)
-        delta_kernel<float, 16><<<grid, kThreads, 0, st>>>(items, (const uint4 *)op, (const uint4 *)gp, dp);
-    else if (dtype == BA_FP32 && lpi == 32)
-        delta_kernel<float, 32><<<grid, kThreads, 0, st>>>(items, (const uint4 *)op, (const uint4 *)gp, dp);
-    else if (dtype == BA_BF16 && lpi == 8)
-        delta_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, st>>>(items, (const uint4 *)op, (const uint4 *)gp, dp);
-    else if (dtype == BA_BF16 && lpi == 16)
-        delta_kernel<__nv_bfloat16, 16><<<grid, kThreads, 0, st>>>(items, (const uint4 *)op, (const uint4 *)gp, dp);
-    else
-        return BA_EUNSUPPORTED;
+#define BA_DELTA_LAUNCH(T, L)                                                                              \
+    delta_kernel<T, L><<<grid, kThreads, 0, st>>>(items, op, gp, lse, delta_t, nlse2_t, row_begin, h_q,   \
+                                                  row_pitch)
+    if (dtype == BA_FP32 && lpi == 16) BA_DELTA_LAUNCH(float, 16);
+    else if (dtype == BA_FP32 && lpi == 32) BA_DELTA_LAUNCH(float, 32);
+    else if (dtype == BA_BF16 && lpi == 8) BA_DELTA_LAUNCH(__nv_bfloat16, 8);
+    else if (dtype == BA_BF16 && lpi == 16) BA_DELTA_LAUNCH(__nv_bfloat16, 16);
+    else return BA_EUNSUPPORTED;
+#undef BA_DELTA_LAUNCH
     return ba_check_launch();
 }
 

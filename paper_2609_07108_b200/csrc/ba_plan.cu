@@ -294,6 +294,7 @@ extern "C" int ba_plan_create(const ba_problem_t *p, void *plan_mem, size_t plan
     pl->scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
     pl->impl = p->impl == BA_IMPL_AUTO ? (ba_tc_supported(p) ? BA_IMPL_TC : BA_IMPL_SIMT) : p->impl;
     pl->pairs = (int64_t)pairs_host;
+    pl->row_pitch = ba_row_pitch(p->n_main + p->n_branch);
     pl->host_offsets = host_offsets;
     pl->dev_status = a.status;
     *out = pl;

@@ -27,7 +27,8 @@ struct SimtArgs {
     BaMeta meta;
     BaRange r;
     const void *q_main, *q_branch, *k, *v, *d_o;
-    const float *lse_in, *delta;
+    const float *lse_in, *delta;  // delta: head-major [h_q, delta_pitch]
+    int64_t delta_pitch;
     void *o;          // forward output
     float *lse_out;
     void *dq_main, *dq_branch, *dk, *dv;
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(kThreads) simt_row_kernel(const SimtArgs a) {
                 go[4 * e] = x.x; go[4 * e + 1] = x.y; go[4 * e + 2] = x.z; go[4 * e + 3] = x.w;
             }
             lse2 = a.lse_in[grow * a.h_q + h] * kLog2e;
-            dlt = a.delta[grow * a.h_q + h];
+            dlt = a.delta[(size_t)h * a.delta_pitch + grow];
         }
     }
     __syncthreads();
@@ -332,7 +333,7 @@ __global__ void __launch_bounds__(kThreads) simt_dkdv_kernel(const SimtArgs a) {
                 load_tile<T, D>(g_s, (const T *)a.d_o, grow0, cnt, a.h_q, h);
                 if (tid < cnt) {
                     lse_s[tid] = a.lse_in[(grow0 + tid) * a.h_q + h] * kLog2e;
-                    dlt_s[tid] = a.delta[(grow0 + tid) * a.h_q + h];
+                    dlt_s[tid] = a.delta[(size_t)h * a.delta_pitch + grow0 + tid];
                     lo_s[tid] = a.meta.row_lo[grow0 + tid];
                     hi_s[tid] = a.meta.row_hi[grow0 + tid];
                     if (phase == 1) {
@@ -456,7 +457,7 @@ int bwd_dispatch(const ba_plan *pl, const BaRange &r, const void *q_main, const 
                  bool do_dq, bool do_dkdv) {
     SimtArgs a = base_args(pl, r);
     a.q_main = q_main; a.q_branch = q_branch; a.k = k; a.v = v; a.d_o = d_o;
-    a.lse_in = lse; a.delta = delta; a.accumulate = accumulate;
+    a.lse_in = lse; a.delta = delta; a.delta_pitch = pl->row_pitch; a.accumulate = accumulate;
     a.dq_main = dq_main; a.dq_branch = dq_branch; a.dk = dk; a.dv = dv;
     const int d = pl->prob.head_dim;
     if (pl->prob.dtype == BA_FP32)

@@ -59,21 +59,25 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // kernels lasts microseconds) or as soon as another thread of the CTA raised
 // `*abort_flag`; then raises the flag itself and returns false, so that every
 // role leaves its loop, the CTA frees its tensor memory and exits cleanly.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// The clock is only looked at every 4096 failed polls (reading a timer on every
+// wait would sit on the critical path of each producer/consumer handoff); the
+// limit is in SM cycles, about two seconds.
+constexpr long long kWaitLimitCycles = 4000000000ll;
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 1023u) == 0) {
+    long long t0 = 0;
+#pragma unroll 1
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 4095u) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
-    return true;
 }
 
 // ----------------------------------------------------------------------- TMA
@@ -89,6 +93,25 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *m, int
         "[%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2),
         "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Ask for a tile / a byte range to be brought into L2 ahead of its load.
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *m, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_prefetch(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes)
+                 : "memory");
+}
+
+// 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
 

@@ -54,7 +54,8 @@ struct DqSmem {
 struct TcBwdParams {
     BaMeta meta;
     BaRange r;
-    const float *lse, *delta;
+    const float *nlse2_t, *delta_t;   // head-major [h_q, row_pitch]: -LSE log2(e), delta
+    int64_t row_pitch;
     void *dq_main, *dq_branch, *dk, *dv;
     int h_q, h_kv, group, pairs_per_group;
     float scale, scale_log2;
@@ -327,8 +328,8 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
         float neg_lse2 = -INFINITY, dlt = 0.f;  // dead rows: P = exp2(-inf) = 0
         if (valid) {
             const int64_t grow = is_main ? my_row : n + my_row;
-            neg_lse2 = -p.lse[grow * p.h_q + h] * kLog2e;
-            dlt = p.delta[grow * p.h_q + h];
+            neg_lse2 = p.nlse2_t[(size_t)h * p.row_pitch + grow];
+            dlt = p.delta_t[(size_t)h * p.row_pitch + grow];
         }
         bool ok = true;
         for (int j = 0; j < T; ++j) {
@@ -500,10 +501,16 @@ __device__ __forceinline__ void quarter_pds(const uint32_t (&rs)[16], const uint
             p1.x = ((mk >> (e + 2)) & 1u) ? p1.x : 0.f;
             p1.y = ((mk >> (e + 3)) & 1u) ? p1.y : 0.f;
         }
-        const float2 d0 = fmul2(p0, fadd2(make_float2(__uint_as_float(rd[e]), __uint_as_float(rd[e + 1])),
-                                          make_float2(-dv.x, -dv.y)));
-        const float2 d1 = fmul2(p1, fadd2(make_float2(__uint_as_float(rd[e + 2]), __uint_as_float(rd[e + 3])),
-                                          make_float2(-dv.z, -dv.w)));
+        float2 d0 = fmul2(p0, fadd2(make_float2(__uint_as_float(rd[e]), __uint_as_float(rd[e + 1])),
+                                    make_float2(-dv.x, -dv.y)));
+        float2 d1 = fmul2(p1, fadd2(make_float2(__uint_as_float(rd[e + 2]), __uint_as_float(rd[e + 3])),
+                                    make_float2(-dv.z, -dv.w)));
+        if (MASKED) {  // the scalars of invisible columns may be anything, even NaN
+            d0.x = ((mk >> e) & 1u) ? d0.x : 0.f;
+            d0.y = ((mk >> (e + 1)) & 1u) ? d0.y : 0.f;
+            d1.x = ((mk >> (e + 2)) & 1u) ? d1.x : 0.f;
+            d1.y = ((mk >> (e + 3)) & 1u) ? d1.y : 0.f;
+        }
         pk[e >> 1] = pack_bf16(p0.x, p0.y);
         pk[(e >> 1) + 1] = pack_bf16(p1.x, p1.y);
         dk8[e >> 1] = pack_bf16(d0.x, d0.y);
@@ -576,7 +583,11 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
-    // ---- query segments: main rows [m0, m1), branch tokens [b0, b1)
+    // ---- query segments: main rows [m0, m1), branch tokens [b0, b1).  Sub-tiles
+    // start at ma / ba: the segment starts moved back (by < 4 rows) so that every
+    // sub-tile's first row is a multiple of 4 in the [N + M] row numbering; this
+    // keeps the bulk copies of the per-row scalars 16-byte aligned.  The extra
+    // leading rows are masked like any other invisible row.
     int64_t m0 = 0, m1 = 0, b0 = 0, b1 = 0;
     if (main_keys && p.has_main_q) {
         m0 = max(key0, p.r.qm_begin);
@@ -586,8 +597,10 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
         b0 = max((int64_t)sm.bq0_min, p.r.tok_begin);
         b1 = min((int64_t)sm.bq1_max, p.r.tok_end);
     }
-    const int n_sub_main = m1 > m0 ? (int)((m1 - m0 + kSub - 1) / kSub) : 0;
-    const int n_sub_br = b1 > b0 ? (int)((b1 - b0 + kSub - 1) / kSub) : 0;
+    const int64_t ma = m0 & ~(int64_t)3;
+    const int64_t ba = ((n + b0) & ~(int64_t)3) - n;   // may be as low as -3
+    const int n_sub_main = m1 > m0 ? (int)((m1 - ma + kSub - 1) / kSub) : 0;
+    const int n_sub_br = b1 > b0 ? (int)((b1 - ba + kSub - 1) / kSub) : 0;
     const int n_sub = n_sub_main + n_sub_br;
     const int n_iter = n_sub * p.group;
 
@@ -603,67 +616,63 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             }
             bool ok = true;
             int issued = 0;
-            // per-row scalars of a sub-tile (2 rows per lane), fetched one
-            // iteration ahead so their latency is off the producer's critical path
-            float nx_lse[2], nx_dl[2];
-            int nx_bs[2];
-            unsigned long long nx_mk[2];
-            auto fetch = [&](int t) {
-                const int h = g * p.group + t / n_sub;
-                const int s = t % n_sub;
-                const bool seg_main = s < n_sub_main;
-                const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
-                const int64_t rend = seg_main ? m1 : b1;
-                const int64_t grow0 = seg_main ? r0 : n + r0;
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int c = lane + 32 * u;
-                    const bool live = r0 + c < rend;
-                    nx_lse[u] = live ? -p.lse[(grow0 + c) * p.h_q + h] * kLog2e : -INFINITY;
-                    nx_dl[u] = live ? p.delta[(grow0 + c) * p.h_q + h] : 0.f;
-                    nx_bs[u] = 0;
-                    nx_mk[u] = 0ull;
-                    if (!main_keys && live) {
-                        nx_bs[u] = p.meta.br_start[r0 + c];
-                        nx_mk[u] = p.meta.br_mask[r0 + c];
-                    }
-                }
-            };
-            fetch(0);
+            int hh = 0, s = 0;  // t = hh * n_sub + s
+            // the query stream comes from HBM: ask for sub-tile t + kPrefetch to be
+            // brought into L2 while sub-tile t is loaded
+            constexpr int kPrefetch = 16;
+            int ph = 0, ps = 0;
+            for (int i = 0; i < kPrefetch; ++i)
+                if (++ps == n_sub) { ps = 0; ++ph; }
             for (int t = 0; t < n_iter; ++t) {
                 const int st = t % kQStages;
                 if (t >= kQStages) ok = mbar_wait(&sm.q_empty[st], ((t / kQStages) - 1) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                const int h = g * p.group + hh;
+                const bool seg_main = s < n_sub_main;
+                const int64_t r0 = seg_main ? ma + (int64_t)s * kSub : ba + (int64_t)(s - n_sub_main) * kSub;
+                const int64_t grow0 = seg_main ? r0 : n + r0;
+                SubMeta &mt = sm.meta[st];
                 if (lane == 0) {
-                    const int h = g * p.group + t / n_sub;
-                    const int s = t % n_sub;
-                    const bool seg_main = s < n_sub_main;
-                    const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
-                    const int64_t grow0 = seg_main ? r0 : n + r0;
                     const CUtensorMap *tq = seg_main ? &tm_q_main : &tm_q_branch;
-                    mbar_expect_tx(&sm.q_full[st], 2 * kSubBytes);
+                    mbar_expect_tx(&sm.q_full[st], 2 * kSubBytes + 2 * kSub * 4);
                     for (int half = 0; half < 2; ++half) {
                         tma_load_3d(sm.qs[st] + half * 8192, tq, half * 64, h, (int)r0, &sm.q_full[st]);
                         tma_load_3d(sm.qs[st] + kSubBytes + half * 8192, &tm_go, half * 64, h, (int)grow0,
                                     &sm.q_full[st]);
                     }
-                }
-                SubMeta &mt = sm.meta[st];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int c = lane + 32 * u;
-                    mt.neg_lse2[c] = nx_lse[u];
-                    mt.delta[c] = nx_dl[u];
-                    if (!main_keys) {
-                        mt.bstart[c] = nx_bs[u];
-                        mt.mask[c] = nx_mk[u];
+                    const size_t off = (size_t)h * p.row_pitch + grow0;
+                    bulk_load(mt.neg_lse2, p.nlse2_t + off, kSub * 4, &sm.q_full[st]);
+                    bulk_load(mt.delta, p.delta_t + off, kSub * 4, &sm.q_full[st]);
+                    if (t + kPrefetch < n_iter) {
+                        const int h2 = g * p.group + ph;
+                        const bool main2 = ps < n_sub_main;
+                        const int64_t r2 = main2 ? ma + (int64_t)ps * kSub : ba + (int64_t)(ps - n_sub_main) * kSub;
+                        const int64_t g2 = main2 ? r2 : n + r2;
+                        const CUtensorMap *tq2 = main2 ? &tm_q_main : &tm_q_branch;
+                        for (int half = 0; half < 2; ++half) {
+                            tma_prefetch_3d(tq2, half * 64, h2, (int)r2);
+                            tma_prefetch_3d(&tm_go, half * 64, h2, (int)g2);
+                        }
+                        const size_t off2 = (size_t)h2 * p.row_pitch + g2;
+                        bulk_prefetch(p.nlse2_t + off2, kSub * 4);
+                        bulk_prefetch(p.delta_t + off2, kSub * 4);
                     }
                 }
-                if (t + 1 < n_iter) fetch(t + 1);
+                if (++ps == n_sub) { ps = 0; ++ph; }
+                if (!main_keys) {
+                    // own-branch tiles (rare, tiny): branch start and mask of each query token
+                    for (int c = lane; c < kSub; c += 32) {
+                        const int64_t tok = r0 + c;
+                        const bool live = tok >= b0 && tok < b1;
+                        mt.bstart[c] = live ? p.meta.br_start[tok] : 0;
+                        mt.mask[c] = live ? p.meta.br_mask[tok] : 0ull;
+                    }
+                }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.q_full[st]);  // second arrival: the scalars are in place
+                if (lane == 0) mbar_arrive(&sm.q_full[st]);  // second arrival: plain stores are in place
                 issued = t + 1;
+                if (++s == n_sub) { s = 0; ++hh; }
             }
             if (!ok && lane == 0) {
                 for (int t = max(issued - kQStages, 0); t < issued; ++t) {
@@ -736,8 +745,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             const int st = t % kQStages;
             const int s = t % n_sub;
             const bool seg_main = s < n_sub_main;
-            const int64_t r0 = seg_main ? m0 + (int64_t)s * kSub : b0 + (int64_t)(s - n_sub_main) * kSub;
-            const int64_t rend = seg_main ? m1 : b1;
+            const int64_t r0 = seg_main ? ma + (int64_t)s * kSub : ba + (int64_t)(s - n_sub_main) * kSub;
+            const int64_t rbeg = seg_main ? m0 : b0, rend = seg_main ? m1 : b1;
             const SubMeta &mt = sm.meta[st];
             // --- which of the 64 query rows (columns) see my key (needs only the
             // stage's scalars, so it runs while the MMAs are still in flight)
@@ -747,12 +756,13 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             if (kvalid) {
                 if (main_keys) {
                     if (seg_main)  // same sequence, causal: key <= row < end of the key's sequence
-                        vis = bit_range((int)(my_key - r0), (int)(min((int64_t)my_qend, rend) - 1 - r0));
+                        vis = bit_range((int)(max((int64_t)my_key, rbeg) - r0), (int)(min((int64_t)my_qend, rend) - 1 - r0));
                     else           // branch tokens anchored at or after the key, inside its sequence
-                        vis = bit_range((int)(my_bq0 - r0), (int)(min((int64_t)my_bq1, rend) - 1 - r0));
+                        vis = bit_range((int)(max((int64_t)my_bq0, rbeg) - r0), (int)(min((int64_t)my_bq1, rend) - 1 - r0));
                 } else {
                     // own-branch tokens whose mask has my bit
-                    const int lo_c = max((int)(my_bq0 - r0), 0), hi_c = min((int)(min((int64_t)my_bq1, rend) - 1 - r0), kSub - 1);
+                    const int lo_c = max((int)(max((int64_t)my_bq0, rbeg) - r0), 0);
+                    const int hi_c = min((int)(min((int64_t)my_bq1, rend) - 1 - r0), kSub - 1);
                     for (int c = lo_c; c <= hi_c; ++c) {
                         const int rel = my_key - mt.bstart[c];
                         if (rel >= 0 && rel < 64 && ((mt.mask[c] >> rel) & 1ull)) vis |= 1ull << c;
@@ -851,8 +861,10 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
     memset(&p, 0, sizeof p);
     p.meta = pl->meta;
     p.r = r;
-    p.lse = lse;
-    p.delta = delta;
+    (void)lse;
+    p.delta_t = delta;
+    p.nlse2_t = delta + (size_t)pl->row_pitch * pr.h_q;
+    p.row_pitch = pl->row_pitch;
     p.dq_main = dq_main; p.dq_branch = dq_branch; p.dk = dk; p.dv = dv;
     p.h_q = pr.h_q; p.h_kv = pr.h_kv;
     p.group = pr.h_q / pr.h_kv;
