@@ -193,8 +193,15 @@ class Recorder:
         return self._wrap("lse_merge", 1, self.ba.lse_merge, *a, **k)
 
     def branch_attn_bwd(self, plan, q_main, *a, **k):
-        # delta (main rows, branch rows) + dQ + dK/dV
-        return self._wrap("bwd", 4 if q_main is not None else 3, self.ba.branch_attn_bwd, plan, q_main, *a, **k)
+        # the three stages of one backward call, bracketed separately:
+        # preprocess (delta of main rows, of branch rows), dQ kernel, dK/dV kernel
+        ba = self.ba
+        out = self._wrap("bwd_prep", 2 if q_main is not None else 1, ba.branch_attn_bwd, plan, q_main, *a,
+                         stages=ba.STAGE_PREP, **k)
+        k2 = dict(k)
+        k2["grads"] = out
+        self._wrap("bwd_dq", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DQ, **k2)
+        return self._wrap("bwd_dkdv", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DKDV, **k2)
 
     def ba_finalize_grads(self, *a, **k):
         return self._wrap("finalize", 1, self.ba.ba_finalize_grads, *a, **k)
@@ -310,13 +317,18 @@ def run_ours(args):
         kind = max(totals, key=lambda k: totals[k][0])
         ms, calls = totals[kind]
         # algorithmic flop of all launches of that kind over the timed steps
-        share = {"fwd": 4.0, "bwd": 10.0}.get(kind)
+        # flop per visible pair and query head that the kernel itself executes, in
+        # units of head_dim: forward 2 GEMMs (QK^T, PV); dQ kernel 3 (S, dP, dQ);
+        # dK/dV kernel 4 (S^T and dP^T recomputed, dV, dK)
+        share = {"fwd": 4.0, "bwd_dq": 6.0, "bwd_dkdv": 8.0}.get(kind)
+        kernel_name = {"fwd": "tc_fwd_kernel", "bwd_dq": "tc_dq_kernel", "bwd_dkdv": "tc_dkdv_kernel"}.get(kind, kind)
         if share is not None:
             kflops = pairs * p.head_dim * p.h_q * share * args.steps
             achieved = kflops / (ms * 1e-3) / 1e12
             long_step = total_ms / args.steps > 1000.0
             peak = peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"]
-            roof = {"bound": "tensor", "kernel": kind, "achieved": round(achieved, 2), "peak": peak,
+            roof = {"bound": "tensor", "kernel": kernel_name, "flop_per_pair_head": share * p.head_dim,
+                    "achieved": round(achieved, 2), "peak": peak,
                     "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": None,
                     "peak_source": f"{peaks['_source']} {'sustained' if long_step else 'burst'} bf16",
                     "launches": calls, "avg_launch_ms": round(ms / calls, 4),
@@ -463,11 +475,20 @@ def time_oracle(p, n_rows, backward=True):
     return fl / dt / 1e12, dt, len(rows), pairs, p1.h_q
 
 
+def sized_rows(p, seconds_target, backward):
+    """Sample size whose oracle run takes about `seconds_target` (found by doubling)."""
+    n_rows, dt = 8, 0.0
+    while n_rows < p.rows:
+        _, dt, _, _, _ = time_oracle(p, n_rows, backward)
+        if dt >= seconds_target / 4:
+            break
+        n_rows *= 4
+    return int(max(8, min(p.rows, n_rows * seconds_target / max(dt, 1e-3))))
+
+
 def cpu_baseline(p, seconds_target=15.0, backward=True):
     cores = len(os.sched_getaffinity(0))
-    # calibrate on a few rows, then size the sample for ~seconds_target
-    _, dt, nr, pairs, _ = time_oracle(p, 4, backward)
-    n_rows = int(max(4, min(p.rows, 4 * seconds_target / max(dt, 1e-3))))
+    n_rows = sized_rows(p, seconds_target, backward)
     val, dt, nr, pairs, hq = time_oracle(p, n_rows, backward)
     return {"value": float(f"{val:.6g}"), "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{nr} uniformly sampled query rows x {hq} query heads of one KV group, "
@@ -482,10 +503,9 @@ def run_reference(args):
     cfg, shrink, cp, backward = WORKLOADS[name]
     p = W.CONFIGS[cfg](shrink)
     cores = len(os.sched_getaffinity(0))
-    _, dt, _, _, _ = time_oracle(p, 4, backward)
-    n_rows = int(max(4, min(p.rows, 4 * args.ref_seconds / max(dt, 1e-3))))
+    n_rows = sized_rows(p, args.ref_seconds, backward)
     for _ in range(args.warmup):
-        time_oracle(p, 4, backward)
+        time_oracle(p, 8, backward)
     vals, secs = [], []
     for _ in range(args.steps):
         val, dt, nr, pairs, hq = time_oracle(p, n_rows, backward)

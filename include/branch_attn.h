@@ -50,6 +50,7 @@ enum { BA_BF16 = 0, BA_FP32 = 1 };
 enum { BA_MASK_CHAIN = 0, BA_MASK_BLOCK = 1, BA_MASK_TREE = 2 };
 enum { BA_PART_MAIN = 1, BA_PART_BRANCH = 2 };
 enum { BA_OP_FWD = 0, BA_OP_BWD = 1 };
+enum { BA_STAGE_PREP = 1, BA_STAGE_DQ = 2, BA_STAGE_DKDV = 4, BA_STAGE_ALL = 7 };
 
 /* Which kernels a plan uses: the tensor-core (tcgen05) path where the shape
  * allows it (bf16, head_dim 128), or the plain-FMA path (any supported shape;
@@ -178,6 +179,23 @@ int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const void *q_bra
                     int64_t kv_begin, int64_t kv_end, int parts, int accumulate,
                     void *dQ_main, void *dQ_branch, void *dK, void *dV,
                     void *workspace, size_t ws_bytes, void *stream);
+
+/*
+ * The same backward, one stage at a time (same arguments, same workspace):
+ *   BA_STAGE_PREP  delta = <dO, O> and -LSE log2(e) of the selected query rows
+ *                  into the workspace (must precede the other two stages),
+ *   BA_STAGE_DQ    dQ of the selected query rows,
+ *   BA_STAGE_DKDV  dK, dV of the selected key set.
+ * `stages` is a bit mask; BA_STAGE_ALL is branch_attn_bwd.  Lets a caller time
+ * or overlap the three kernels separately.
+ */
+int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                           const void *k, const void *v, const void *O, const float *LSE,
+                           const void *dO,
+                           int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                           int64_t kv_begin, int64_t kv_end, int parts, int accumulate,
+                           void *dQ_main, void *dQ_branch, void *dK, void *dV,
+                           void *workspace, size_t ws_bytes, void *stream, int stages);
 
 /* fp32 accumulators -> dst_dtype (round to nearest even), `count` elements. */
 int ba_finalize_grads(const float *src, void *dst, int64_t count, int dst_dtype, void *stream);

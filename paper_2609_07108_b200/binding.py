@@ -18,6 +18,7 @@ from . import build as _build
 BA_BF16, BA_FP32 = 0, 1
 PART_MAIN, PART_BRANCH, PART_ALL = 1, 2, 3
 OP_FWD, OP_BWD = 0, 1
+STAGE_PREP, STAGE_DQ, STAGE_DKDV, STAGE_ALL = 1, 2, 4, 7
 IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
 
 _DT = {"bf16": (BA_BF16, torch.bfloat16), "fp32": (BA_FP32, torch.float32)}
@@ -45,7 +46,8 @@ class _Problem(C.Structure):
 _LIB = None
 EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
            "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "ba_plan_check", "branch_attn_fwd",
-           "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd", "ba_finalize_grads")
+           "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd", "branch_attn_bwd_stages",
+           "ba_finalize_grads")
 
 
 def _lib():
@@ -86,6 +88,8 @@ def _lib():
         lib.branch_attn_bwd.restype = C.c_int
         lib.branch_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64,
                                         C.c_int, C.c_int, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        lib.branch_attn_bwd_stages.restype = C.c_int
+        lib.branch_attn_bwd_stages.argtypes = lib.branch_attn_bwd.argtypes + [C.c_int]
         lib.ba_finalize_grads.restype = C.c_int
         lib.ba_finalize_grads.argtypes = [vp, vp, i64, C.c_int, vp]
         _LIB = lib
@@ -231,7 +235,7 @@ def lse_merge(o_a, lse_a, o_b, lse_b, out=None, lse_out=None, out_dtype=torch.fl
 
 
 def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br_range=None,
-                    kv_range=None, parts=PART_ALL, accumulate=False, grads=None):
+                    kv_range=None, parts=PART_ALL, accumulate=False, grads=None, stages=STAGE_ALL):
     """(dQ_main, dQ_branch, dK, dV).  With `accumulate`, `grads` must hold four
     zero-initialised fp32 tensors which receive the selected terms."""
     p = plan.problem
@@ -247,11 +251,14 @@ def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br
                  mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device),
                  mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device))
     ws = plan.workspace(OP_BWD)
-    rc = _lib().branch_attn_bwd(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(o), _p(lse),
-                                _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1],
-                                kv_range[0], kv_range[1], parts, 1 if accumulate else 0,
-                                _p(grads[0]), _p(grads[1]), _p(grads[2]), _p(grads[3]),
-                                _p(ws), ws.numel(), _stream())
+    args = (plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(o), _p(lse),
+            _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1],
+            kv_range[0], kv_range[1], parts, 1 if accumulate else 0,
+            _p(grads[0]), _p(grads[1]), _p(grads[2]), _p(grads[3]), _p(ws), ws.numel(), _stream())
+    if stages == STAGE_ALL:
+        rc = _lib().branch_attn_bwd(*args)
+    else:
+        rc = _lib().branch_attn_bwd_stages(*args, stages)
     _check(rc, "branch_attn_bwd")
     return grads
 

@@ -88,7 +88,19 @@ extern "C" int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const 
                                int64_t br_end, int64_t kv_begin, int64_t kv_end, int parts,
                                int accumulate, void *dQ_main, void *dQ_branch, void *dK, void *dV,
                                void *workspace, size_t ws_bytes, void *stream) {
+    return branch_attn_bwd_stages(plan, q_main, q_branch, k, v, O, LSE, dO, qm_begin, qm_end, br_begin, br_end,
+                                  kv_begin, kv_end, parts, accumulate, dQ_main, dQ_branch, dK, dV, workspace,
+                                  ws_bytes, stream, BA_STAGE_ALL);
+}
+
+extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                                      const void *k, const void *v, const void *O, const float *LSE,
+                                      const void *dO, int64_t qm_begin, int64_t qm_end, int64_t br_begin,
+                                      int64_t br_end, int64_t kv_begin, int64_t kv_end, int parts,
+                                      int accumulate, void *dQ_main, void *dQ_branch, void *dK, void *dV,
+                                      void *workspace, size_t ws_bytes, void *stream, int stages) {
     if (!plan) return BA_EINVAL;
+    if (stages <= 0 || stages > BA_STAGE_ALL) return BA_EINVAL;
     BaRange r;
     int rc = make_range(plan, qm_begin, qm_end, br_begin, br_end, kv_begin, kv_end, parts, &r);
     if (rc != BA_OK) return rc;
@@ -108,14 +120,19 @@ extern "C" int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const 
     const int64_t rp = plan->row_pitch;
     const int64_t n = plan->prob.n_main;
     const int hq = plan->prob.h_q, d = plan->prob.head_dim, dt = plan->prob.dtype;
-    if (has_main_q && (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, r.qm_begin, r.qm_end, hq, d, dt, st)) != BA_OK) return rc;
-    if (has_branch_q &&
-        (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
-        return rc;
+    if (stages & BA_STAGE_PREP) {
+        if (has_main_q &&
+            (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, r.qm_begin, r.qm_end, hq, d, dt, st)) != BA_OK)
+            return rc;
+        if (has_branch_q &&
+            (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
+            return rc;
+    }
+    if (!(stages & (BA_STAGE_DQ | BA_STAGE_DKDV))) return BA_OK;
     const void *qm = has_main_q ? q_main : nullptr;
     if (plan->impl == BA_IMPL_TC)
         return ba_tc_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK,
-                         dV, st);
+                         dV, st, stages);
     return ba_simt_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK, dV,
-                       st);
+                       st, stages);
 }

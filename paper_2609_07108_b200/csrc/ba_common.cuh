@@ -68,10 +68,7 @@ int ba_simt_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const v
 int ba_simt_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
                 const void *k, const void *v, const float *lse, const float *delta,
                 const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
-                void *dv, cudaStream_t st);
-int ba_simt_bwd_dkdv(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
-                     const void *k, const void *v, const float *lse, const float *delta,
-                     const void *d_o, int accumulate, void *dk, void *dv, cudaStream_t st);
+                void *dv, cudaStream_t st, int stages);
 // Tensor-core path (ba_tc_fwd.cu / ba_tc_bwd.cu)
 int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
               const void *k, const void *v, void *o, float *lse, bool partial_out,
@@ -79,7 +76,7 @@ int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
 int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
               const void *k, const void *v, const float *lse, const float *delta,
               const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
-              void *dv, cudaStream_t st);
+              void *dv, cudaStream_t st, int stages);
 bool ba_tc_supported(const ba_problem_t *p);
 // Elementwise (ba_elementwise.cu)
 // Backward preprocess into head-major scratch [h_q, row_pitch]:

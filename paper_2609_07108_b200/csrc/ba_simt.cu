@@ -482,14 +482,7 @@ int ba_simt_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const v
 int ba_simt_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
                 const void *k, const void *v, const float *lse, const float *delta,
                 const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
-                void *dv, cudaStream_t st) {
+                void *dv, cudaStream_t st, int stages) {
     return bwd_dispatch(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, dq_main, dq_branch, dk, dv,
-                        st, true, true);
-}
-
-int ba_simt_bwd_dkdv(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
-                     const void *k, const void *v, const float *lse, const float *delta,
-                     const void *d_o, int accumulate, void *dk, void *dv, cudaStream_t st) {
-    return bwd_dispatch(pl, r, q_main, q_branch, k, v, lse, delta, d_o, accumulate, nullptr, nullptr, dk, dv,
-                        st, false, true);
+                        st, (stages & BA_STAGE_DQ) != 0, (stages & BA_STAGE_DKDV) != 0);
 }

@@ -847,7 +847,7 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
 
 int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
               const void *v, const float *lse, const float *delta, const void *d_o, int accumulate,
-              void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st) {
+              void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st, int stages) {
     static bool attr_set = false;
     const size_t dq_smem = sizeof(DqSmem) + 1024;
     const size_t kv_smem = sizeof(KvSmem) + 1024;
@@ -892,7 +892,7 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
         !make_tmap_rhd(&tq_branch, qb, qb_rows, pr.h_q, 128, kTile))
         return BA_EINVAL;
 
-    if (p.total_tiles > 0) {
+    if (p.total_tiles > 0 && (stages & BA_STAGE_DQ)) {
         const int64_t grid = (int64_t)p.total_tiles * pr.h_kv * p.pairs_per_group;
         if (grid > INT_MAX) return BA_EUNSUPPORTED;
         tc_dq_kernel<<<(unsigned)grid, kDqThreads, dq_smem, st>>>(tq_main, tq_branch, tgo, tk, tv, p);
@@ -904,7 +904,7 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
     const int64_t kbt = (r.parts & BA_PART_BRANCH) ? (r.tok_end - r.tok_begin + kTile - 1) / kTile : 0;
     p.main_key_tiles = (int)kmt;
     p.total_key_tiles = (int)(kmt + kbt);
-    if (p.total_key_tiles > 0) {
+    if (p.total_key_tiles > 0 && (stages & BA_STAGE_DKDV)) {
         CUtensorMap tq_main64, tq_branch64, tgo64;
         if (!make_tmap_rhd(&tq_main64, qm, qm_rows, pr.h_q, 128, kSub) ||
             !make_tmap_rhd(&tq_branch64, qb, qb_rows, pr.h_q, 128, kSub) ||
