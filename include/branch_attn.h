@@ -197,6 +197,38 @@ int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main, const void
                            void *dQ_main, void *dQ_branch, void *dK, void *dV,
                            void *workspace, size_t ws_bytes, void *stream, int stages);
 
+/*
+ * Backward without caller-provided scratch.  (No counterpart in the paper: this
+ * is a packaging variant of branch_attn_bwd, same arithmetic, same results.)
+ *
+ * For callers that cannot allocate device memory when they call -- code running
+ * inside a fixed, pre-planned memory arena, or under a framework hook where
+ * allocator calls are forbidden -- and so have nothing to pass as `workspace`.
+ * The per-row scalars of the backward (delta and -LSE log2 e) are kept in an
+ * array of BA_STATIC_SCRATCH_BYTES that is part of the library image; every GPU
+ * that loads the library holds that much memory until the process exits.
+ *   - Arguments are those of branch_attn_bwd without workspace / ws_bytes; the
+ *     caller still owns all inputs and outputs.
+ *   - Limit: ba_workspace_bytes(plan, BA_OP_BWD) must not exceed
+ *     BA_STATIC_SCRATCH_BYTES (8 MiB: 2 * h_q * (N + M + 128, rounded up to 64)
+ *     floats, e.g. 32 query heads and up to 32,640 rows); larger problems get
+ *     BA_EWORKSPACE and nothing is launched.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *     No call allocates or frees device memory.
+ *   - All calls on a device share the one array, which keeps whatever the last
+ *     call left in it.  Nothing in it needs clearing (each call rewrites every
+ *     entry it reads), but two calls whose kernels overlap in time on the GPU --
+ *     different streams, or different host threads -- race on it: serialise them.
+ */
+#define BA_STATIC_SCRATCH_BYTES (8u << 20)
+int branch_attn_bwd_static(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                           const void *k, const void *v, const void *O, const float *LSE,
+                           const void *dO,
+                           int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                           int64_t kv_begin, int64_t kv_end, int parts, int accumulate,
+                           void *dQ_main, void *dQ_branch, void *dK, void *dV, void *stream);
+
 /* fp32 accumulators -> dst_dtype (round to nearest even), `count` elements. */
 int ba_finalize_grads(const float *src, void *dst, int64_t count, int dst_dtype, void *stream);
 

@@ -47,7 +47,7 @@ _LIB = None
 EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
            "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "ba_plan_check", "branch_attn_fwd",
            "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd", "branch_attn_bwd_stages",
-           "ba_finalize_grads")
+           "branch_attn_bwd_static", "ba_finalize_grads")
 
 
 def _lib():
@@ -90,6 +90,8 @@ def _lib():
                                         C.c_int, C.c_int, vp, vp, vp, vp, vp, C.c_size_t, vp]
         lib.branch_attn_bwd_stages.restype = C.c_int
         lib.branch_attn_bwd_stages.argtypes = lib.branch_attn_bwd.argtypes + [C.c_int]
+        lib.branch_attn_bwd_static.restype = C.c_int
+        lib.branch_attn_bwd_static.argtypes = lib.branch_attn_bwd.argtypes[:-3] + [vp]
         lib.ba_finalize_grads.restype = C.c_int
         lib.ba_finalize_grads.argtypes = [vp, vp, i64, C.c_int, vp]
         _LIB = lib
@@ -260,6 +262,30 @@ def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br
     else:
         rc = _lib().branch_attn_bwd_stages(*args, stages)
     _check(rc, "branch_attn_bwd")
+    return grads
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def branch_attn_bwd_static(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br_range=None,
+                           kv_range=None, parts=PART_ALL, accumulate=False, grads=None):
+    """branch_attn_bwd for callers that cannot allocate device scratch at call
+    time: the library's built-in 8 MiB array serves as workspace (problems whose
+    backward scratch is larger raise BA_EWORKSPACE).  `grads` must be given: this
+    wrapper allocates nothing either.  Calls that may overlap on the GPU must be
+    serialised by the caller, they share the one array."""
+    p = plan.problem
+    qm_range = (0, p.n_main) if qm_range is None else qm_range
+    br_range = (0, p.num_branches) if br_range is None else br_range
+    kv_range = (0, p.n_main) if kv_range is None else kv_range
+    if grads is None:
+        raise ValueError("branch_attn_bwd_static writes into caller-provided gradient tensors")
+    rc = _lib().branch_attn_bwd_static(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(o), _p(lse),
+                                       _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1],
+                                       kv_range[0], kv_range[1], parts, 1 if accumulate else 0,
+                                       _p(grads[0]), _p(grads[1]), _p(grads[2]), _p(grads[3]), _stream())
+    _check(rc, "branch_attn_bwd_static")
     return grads
 
 

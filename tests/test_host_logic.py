@@ -82,6 +82,7 @@ def test_library_exports_every_declared_symbol():
     lib = ctypes.CDLL(lib_path)
     header = open(os.path.join(ROOT, "include", "branch_attn.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    header = re.sub(r"^\s*#.*$", "", header, flags=re.M)      # preprocessor lines declare no symbols
     names = re.findall(r"\b([A-Za-z_][A-Za-z0-9_]*)\s*\([^;{]*\)\s*;", header)
     assert {"branch_attn_fwd", "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd",
             "ba_plan_create", "ba_plan_bytes", "ba_finalize_grads"} <= set(names)
