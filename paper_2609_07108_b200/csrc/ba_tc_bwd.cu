@@ -848,13 +848,17 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
 int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
               const void *v, const float *lse, const float *delta, const void *d_o, int accumulate,
               void *dq_main, void *dq_branch, void *dk, void *dv, cudaStream_t st, int stages) {
-    static bool attr_set = false;
+    // the dynamic shared-memory limit is a per-device attribute of the kernel
+    static bool attr_set[64] = {};
+    int dev = 0;
+    BA_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return BA_EUNSUPPORTED;
     const size_t dq_smem = sizeof(DqSmem) + 1024;
     const size_t kv_smem = sizeof(KvSmem) + 1024;
-    if (!attr_set) {
+    if (!attr_set[dev]) {
         BA_CUDA_CHECK(cudaFuncSetAttribute(tc_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dq_smem));
         BA_CUDA_CHECK(cudaFuncSetAttribute(tc_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kv_smem));
-        attr_set = true;
+        attr_set[dev] = true;
     }
     const ba_problem_t &pr = pl->prob;
     TcBwdParams p;

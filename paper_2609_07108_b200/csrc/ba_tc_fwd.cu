@@ -474,11 +474,15 @@ bool ba_tc_supported(const ba_problem_t *p) {
 
 int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
               const void *v, void *o, float *lse, bool partial_out, cudaStream_t st) {
-    static bool attr_set = false;
+    // the dynamic shared-memory limit is a per-device attribute of the kernel
+    static bool attr_set[64] = {};
+    int dev = 0;
+    BA_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return BA_EUNSUPPORTED;
     const size_t smem = sizeof(FwdSmem) + 1024;
-    if (!attr_set) {
+    if (!attr_set[dev]) {
         BA_CUDA_CHECK(cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set = true;
+        attr_set[dev] = true;
     }
     const ba_problem_t &pr = pl->prob;
     TcFwdParams p;

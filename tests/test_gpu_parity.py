@@ -144,6 +144,36 @@ def test_shrunken_configs_bf16(ba, oracle, cfg, shrink):
         check_full(ba, oracle, p, seed=0, std=0.5, impl=impl, backward=(cfg != 2), groups=[0, p.h_kv - 1])
 
 
+@pytest.mark.parametrize("h_q,h_kv", [(2, 2), (3, 1), (5, 1), (6, 2)])
+def test_head_group_sizes(ba, oracle, h_q, h_kv):
+    """Query heads per KV head 1, 3, 5 (an odd head is left over in the head-pair
+    work split of the tensor-core kernels) and 3 again with two KV heads."""
+    p = W.odd_shapes(W.BLOCK, head_dim=128, dtype="bf16", h_q=h_q, h_kv=h_kv)
+    for impl in impls_for(ba, p):
+        check_full(ba, oracle, p, seed=8, std=0.5, impl=impl)
+
+
+def test_branch_part_as_its_own_partial_merged_last(ba, oracle):
+    """The paper's literal order: main-sequence partials over key chunks first,
+    the locally computed branch component merged at the end (Eq. lse-merge)."""
+    p = W.odd_shapes(W.CHAIN, head_dim=128, dtype="bf16")
+    t = W.make_tensors(p, seed=9, std=0.5)
+    d = to_dev(p, t)
+    n, a = p.n_main, p.num_branches
+    for impl in impls_for(ba, p):
+        plan = ba.Plan(p, impl=impl)
+        o_full, lse_full = ba.branch_attn_fwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"])
+        acc = None
+        for kv, parts in (((0, 200), ba.PART_MAIN), ((200, n), ba.PART_MAIN), ((0, 0), ba.PART_BRANCH)):
+            part = ba.branch_attn_fwd_partial(plan, d["q_main"], d["q_branch"], d["k"], d["v"], (0, n), (0, a), kv, parts)
+            acc = part if acc is None else ba.lse_merge(acc[0], acc[1], part[0], part[1])
+        assert_close("merged O", f32(acc[0]), f32(o_full).astype(np.float64), TOL["bf16"])
+        assert_lse_close(f32(acc[1]), f32(lse_full).astype(np.float64))
+        ref = oracle_fwd_bwd(oracle, p, t, backward=False)
+        assert_close("merged O vs oracle", f32(acc[0]), ref["o"], TOL["bf16"])
+        plan.check()
+
+
 def test_no_branches(ba, oracle):
     cu = W.cu_from_lengths([100, 300, 29])
     p = W.Problem(cu, np.zeros(0, np.int32), np.zeros(1, np.int32), W.CHAIN, None, 4, 2, 128, dtype="bf16")
