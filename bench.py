@@ -45,8 +45,8 @@ WORKLOADS = {
 }
 
 
-def useful_flops(p, backward=True):
-    pairs = W.useful_pairs(p)
+def useful_flops(p, backward=True, branch_only=False):
+    pairs = W.useful_pairs(p, with_main_queries=not branch_only)
     per_pair = 4 * p.head_dim * p.h_q
     return pairs * per_pair * (3.5 if backward else 1.0), pairs
 
@@ -261,13 +261,19 @@ def run_ours(args):
     p = W.CONFIGS[cfg](shrink) if cfg != 1 else W.config1()
     impl = {"auto": ba.IMPL_AUTO, "simt": ba.IMPL_SIMT, "tc": ba.IMPL_TC}[args.kernels]
     plan = ba.Plan(p, device=device, impl=impl)
-    flops, pairs = useful_flops(p, backward)
+    branch_only = bool(args.branch_only)
+    if branch_only and cp:
+        raise SystemExit("--branch-only applies to the monolithic workloads")
+    flops, pairs = useful_flops(p, backward, branch_only)
     t = make_device_inputs(p, torch, device)
+    if branch_only:
+        t["q_main"] = None   # draft-only form: main K/V are keys, only branch tokens are queries
     if not cp:
         t["_o"] = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
         t["_lse"] = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=device)
     rec = Recorder(ba, p)
-    in_bytes = sum(t[k].numel() * t[k].element_size() for k in ("q_main", "q_branch", "k", "v", "d_o"))
+    in_bytes = sum(t[k].numel() * t[k].element_size() for k in ("q_main", "q_branch", "k", "v", "d_o")
+                   if t[k] is not None)
     flush = None
     if in_bytes < 512 << 20:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
@@ -353,7 +359,8 @@ def run_ours(args):
                        "head_dim": p.head_dim, "mask": W.KIND_NAMES[p.kind], "pairs_per_head": pairs,
                        "path": (f"zigzag cp={cp}: partial fwd + lse_merge, partial bwd accumulate"
                                 if cp else "monolithic fwd + bwd"),
-                       "backward": backward, "kernels": {ba.IMPL_SIMT: "simt", ba.IMPL_TC: "tcgen05"}[plan.impl],
+                       "backward": backward, "queries": "branch tokens only" if branch_only else "main + branch",
+                       "kernels": {ba.IMPL_SIMT: "simt", ba.IMPL_TC: "tcgen05"}[plan.impl],
                        "l2": "inputs larger than L2" if flush is None else "256 MiB flush between steps",
                        "parallelism": "replicas" if world > 1 else "single"},
             "frac_of_peak": {"burst": round(value / world / peaks["bf16_tflops"], 4),
@@ -376,12 +383,13 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     """Same step, inputs in pinned host memory: H2D of Q/K/V/dO, the library
     calls, D2H of O/LSE and the gradients, all inside the timed region."""
     import psutil
-    names = ("q_main", "q_branch", "k", "v") + (("d_o",) if backward else ())
+    names = tuple(k for k in ("q_main", "q_branch", "k", "v") + (("d_o",) if backward else ()) if t[k] is not None)
     h2d = sum(t[k].numel() * t[k].element_size() for k in names)
     out_shapes = [((p.rows, p.h_q, p.head_dim), plan.torch_dtype), ((p.rows, p.h_q), torch.float32)]
     if backward:
-        out_shapes += [((p.n_main, p.h_q, p.head_dim), plan.torch_dtype),
-                       ((p.n_branch, p.h_q, p.head_dim), plan.torch_dtype),
+        if t["q_main"] is not None:
+            out_shapes += [((p.n_main, p.h_q, p.head_dim), plan.torch_dtype)]
+        out_shapes += [((p.n_branch, p.h_q, p.head_dim), plan.torch_dtype),
                        ((p.rows, p.h_kv, p.head_dim), plan.torch_dtype),
                        ((p.rows, p.h_kv, p.head_dim), plan.torch_dtype)]
     d2h = sum(int(np.prod(s)) * torch.empty(0, dtype=d).element_size() for s, d in out_shapes)
@@ -434,6 +442,7 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
             h2d_copy(t[k], k)
         o, lse, grads = run_step(rec, plan, t, cp, backward)
         outs = [o, lse] + (list(grads[:4]) if backward else [])
+        outs = [x for x in outs if x is not None]
         for i, src in enumerate(outs):
             d2h_copy(i, src)
     e_ev.record()
@@ -567,6 +576,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="auto", choices=["auto", *WORKLOADS])
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--branch-only", action="store_true",
+                    help="q_main = NULL: only the branch tokens are queries (monolithic workloads)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
