@@ -527,8 +527,11 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile int *abort_flag = &sm.abort_flag;
 
-    const int tile = (int)(blockIdx.x / p.h_kv);
-    const int g = (int)(blockIdx.x % p.h_kv);
+    // KV-head-major order: the CTAs resident at one time belong to one or two KV
+    // heads and stream the same query rows, so that stream is read from HBM about
+    // once per head instead of once per wave of CTAs
+    const int g = (int)(blockIdx.x / p.total_key_tiles);
+    const int tile = (int)(blockIdx.x % p.total_key_tiles);
     const bool main_keys = tile < p.main_key_tiles;
     const int64_t n = p.meta.n_main;
     // first key of the tile: main key index, or branch token index
