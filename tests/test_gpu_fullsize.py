@@ -182,3 +182,42 @@ def test_zigzag_equals_monolithic_small(ba):
     for a, b in zip(g1, g2[:4]):
         assert float((a.float() - b.float()).abs().max()) <= 2e-2
     plan.check()
+
+
+def test_config3_full_size_dense_cotangent_one_group(ba, oracle):
+    """Dense dO at full size: every gradient of one KV-head group of the
+    32,768-token DFlash batch against the oracle (all rows, all keys)."""
+    p = W.config3()
+    plan = ba.Plan(p, impl=ba.IMPL_TC)
+    t = device_inputs(p, 11)
+    o, lse = ba.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"])
+    dqm, dqb, dk, dv = ba.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"])
+    plan.check()
+    p2, qh, kvh = head_slice(p, [4])
+    qh_t = torch.from_numpy(qh).cuda()
+    q_all = np.concatenate([f32(t["q_main"][:, qh_t]), f32(t["q_branch"][:, qh_t])], 0)
+    k_h, v_h = f32(t["k"][:, 4:5]), f32(t["v"][:, 4:5])
+    ref_o, ref_lse = oracle.forward(p2, q_all, k_h, v_h)
+    ref_dq, ref_dk, ref_dv = oracle.backward(p2, q_all, k_h, v_h, f32(t["d_o"][:, qh_t]))
+    tol = TOL["bf16"]
+    assert_close("O", f32(o[:, qh_t]), ref_o, tol)
+    assert_lse_close(f32(lse[:, qh_t]), ref_lse)
+    assert_close("dQ", f32(torch.cat([dqm, dqb], 0)[:, qh_t]), ref_dq, tol)
+    assert_close("dK", f32(dk[:, 4:5]), ref_dk, tol)
+    assert_close("dV", f32(dv[:, 4:5]), ref_dv, tol)
+
+
+def test_results_are_bit_identical_from_run_to_run(ba):
+    """Every output element has one owning CTA and a fixed summation order."""
+    p = W.config4(shrink=8)
+    plan = ba.Plan(p, impl=ba.IMPL_TC)
+    t = device_inputs(p, 12)
+    runs = []
+    for _ in range(2):
+        o, lse = ba.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"])
+        g = ba.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"])
+        runs.append((o, lse, *g))
+    torch.cuda.synchronize()
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+    plan.check()
