@@ -168,7 +168,7 @@ class Recorder:
         self.events = []           # (kind, start, end)
         self.launches = 0
         self.enabled = False
-        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL"):
+        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL", "STAGE_ALL", "STAGE_ALL_FUSED"):
             setattr(self, name, getattr(ba, name))
 
     def _wrap(self, kind, n_launch, fn, *a, **k):
@@ -196,10 +196,14 @@ class Recorder:
         # the three stages of one backward call, bracketed separately:
         # preprocess (delta of main rows, of branch rows), dQ kernel, dK/dV kernel
         ba = self.ba
+        k = dict(k)
+        fused = k.pop("stages", ba.STAGE_ALL) == ba.STAGE_ALL_FUSED
         out = self._wrap("bwd_prep", 2 if q_main is not None else 1, ba.branch_attn_bwd, plan, q_main, *a,
                          stages=ba.STAGE_PREP, **k)
         k2 = dict(k)
         k2["grads"] = out
+        if fused:   # one kernel for dQ, dK and dV
+            return self._wrap("bwd_fused", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_FUSED, **k2)
         self._wrap("bwd_dq", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DQ, **k2)
         return self._wrap("bwd_dkdv", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DKDV, **k2)
 
@@ -230,13 +234,13 @@ def make_device_inputs(p, torch, device, seed=0):
     return t
 
 
-def run_step(rec, plan, t, cp, backward):
+def run_step(rec, plan, t, cp, backward, fused=False):
     from paper_2609_07108_b200 import zigzag
     if cp:
         o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp,
                                    out=t.get("_o"), lse=t.get("_lse"))
-        grads = zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp) \
-            if backward else None
+        grads = zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp,
+                                fused=fused) if backward else None
     else:
         o, lse = rec.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"],
                                      out=t.get("_o"), lse=t.get("_lse"))
@@ -283,8 +287,10 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the one-kernel backward adds into fp32 accumulators: the chunked (zigzag) path has them
+    fused = args.bwd == "fused" and bool(cp) and plan.impl == ba.IMPL_TC
     for _ in range(args.warmup):
-        run_step(rec, plan, t, cp, backward)
+        run_step(rec, plan, t, cp, backward, fused=fused)
         if flush is not None:
             flush.fill_(1)
     barrier()
@@ -300,7 +306,7 @@ def run_ours(args):
         s = torch.cuda.Event(enable_timing=True)
         e = torch.cuda.Event(enable_timing=True)
         s.record()
-        run_step(rec, plan, t, cp, backward)
+        run_step(rec, plan, t, cp, backward, fused=fused)
         e.record()
         step_ms.append((s, e))
     barrier()
@@ -326,8 +332,9 @@ def run_ours(args):
         # flop per visible pair and query head that the kernel itself executes, in
         # units of head_dim: forward 2 GEMMs (QK^T, PV); dQ kernel 3 (S, dP, dQ);
         # dK/dV kernel 4 (S^T and dP^T recomputed, dV, dK)
-        share = {"fwd": 4.0, "bwd_dq": 6.0, "bwd_dkdv": 8.0}.get(kind)
-        kernel_name = {"fwd": "tc_fwd_kernel", "bwd_dq": "tc_dq_kernel", "bwd_dkdv": "tc_dkdv_kernel"}.get(kind, kind)
+        share = {"fwd": 4.0, "bwd_dq": 6.0, "bwd_dkdv": 8.0, "bwd_fused": 10.0}.get(kind)
+        kernel_name = {"fwd": "tc_fwd_kernel", "bwd_dq": "tc_dq_kernel", "bwd_dkdv": "tc_dkdv_kernel",
+                       "bwd_fused": "tc_bwd_fused_kernel"}.get(kind, kind)
         if share is not None:
             kflops = pairs * p.head_dim * p.h_q * share * args.steps
             achieved = kflops / (ms * 1e-3) / 1e12
@@ -359,7 +366,10 @@ def run_ours(args):
                        "head_dim": p.head_dim, "mask": W.KIND_NAMES[p.kind], "pairs_per_head": pairs,
                        "path": (f"zigzag cp={cp}: partial fwd + lse_merge, partial bwd accumulate"
                                 if cp else "monolithic fwd + bwd"),
-                       "backward": backward, "queries": "branch tokens only" if branch_only else "main + branch",
+                       "backward": backward,
+                       "bwd_kernels": ("one fused kernel (dQ by fp32 atomic adds)" if fused
+                                       else "dQ kernel + dK/dV kernel") if backward else None,
+                       "queries": "branch tokens only" if branch_only else "main + branch",
                        "kernels": {ba.IMPL_SIMT: "simt", ba.IMPL_TC: "tcgen05"}[plan.impl],
                        "l2": "inputs larger than L2" if flush is None else "256 MiB flush between steps",
                        "parallelism": "replicas" if world > 1 else "single"},
@@ -440,7 +450,7 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     for _ in range(steps):
         for k in names:
             h2d_copy(t[k], k)
-        o, lse, grads = run_step(rec, plan, t, cp, backward)
+        o, lse, grads = run_step(rec, plan, t, cp, backward, fused=args.bwd == "fused" and bool(cp))
         outs = [o, lse] + (list(grads[:4]) if backward else [])
         outs = [x for x in outs if x is not None]
         for i, src in enumerate(outs):
@@ -576,6 +586,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="auto", choices=["auto", *WORKLOADS])
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--bwd", default="split", choices=["split", "fused"],
+                    help="backward of the chunked workloads: dQ kernel + dK/dV kernel, or one kernel "
+                         "for all three (dQ summed with atomic adds)")
     ap.add_argument("--branch-only", action="store_true",
                     help="q_main = NULL: only the branch tokens are queries (monolithic workloads)")
     ap.add_argument("--no-e2e", action="store_true")

@@ -50,7 +50,8 @@ enum { BA_BF16 = 0, BA_FP32 = 1 };
 enum { BA_MASK_CHAIN = 0, BA_MASK_BLOCK = 1, BA_MASK_TREE = 2 };
 enum { BA_PART_MAIN = 1, BA_PART_BRANCH = 2 };
 enum { BA_OP_FWD = 0, BA_OP_BWD = 1 };
-enum { BA_STAGE_PREP = 1, BA_STAGE_DQ = 2, BA_STAGE_DKDV = 4, BA_STAGE_ALL = 7 };
+enum { BA_STAGE_PREP = 1, BA_STAGE_DQ = 2, BA_STAGE_DKDV = 4, BA_STAGE_ALL = 7,
+       BA_STAGE_FUSED = 8, BA_STAGE_ALL_FUSED = 9 };
 
 /* Which kernels a plan uses: the tensor-core (tcgen05) path where the shape
  * allows it (bf16, head_dim 128), or the plain-FMA path (any supported shape;
@@ -188,6 +189,14 @@ int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const void *q_bra
  *   BA_STAGE_DKDV  dK, dV of the selected key set.
  * `stages` is a bit mask; BA_STAGE_ALL is branch_attn_bwd.  Lets a caller time
  * or overlap the three kernels separately.
+ *   BA_STAGE_FUSED replaces BA_STAGE_DQ | BA_STAGE_DKDV (it cannot be combined
+ *                  with them) by ONE key-stationary kernel that forms S and dP
+ *                  once per tile pair (10 D flop per visible pair instead of 14 D)
+ *                  and sums dQ into its fp32 accumulator with atomic adds.
+ *                  Needs accumulate = 1 and the tensor-core kernels, else
+ *                  BA_EUNSUPPORTED.  dK and dV stay bit-reproducible; the last
+ *                  bits of dQ depend on the order in which the key tiles arrive.
+ *   BA_STAGE_ALL_FUSED = BA_STAGE_PREP | BA_STAGE_FUSED.
  */
 int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main, const void *q_branch,
                            const void *k, const void *v, const void *O, const float *LSE,

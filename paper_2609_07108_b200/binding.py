@@ -19,6 +19,7 @@ BA_BF16, BA_FP32 = 0, 1
 PART_MAIN, PART_BRANCH, PART_ALL = 1, 2, 3
 OP_FWD, OP_BWD = 0, 1
 STAGE_PREP, STAGE_DQ, STAGE_DKDV, STAGE_ALL = 1, 2, 4, 7
+STAGE_FUSED, STAGE_ALL_FUSED = 8, 9
 IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
 
 _DT = {"bf16": (BA_BF16, torch.bfloat16), "fp32": (BA_FP32, torch.float32)}

@@ -100,7 +100,8 @@ extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main,
                                       int accumulate, void *dQ_main, void *dQ_branch, void *dK, void *dV,
                                       void *workspace, size_t ws_bytes, void *stream, int stages) {
     if (!plan) return BA_EINVAL;
-    if (stages <= 0 || stages > BA_STAGE_ALL) return BA_EINVAL;
+    if (stages <= 0 || stages > (BA_STAGE_ALL | BA_STAGE_FUSED)) return BA_EINVAL;
+    if ((stages & BA_STAGE_FUSED) && (stages & (BA_STAGE_DQ | BA_STAGE_DKDV))) return BA_EINVAL;
     BaRange r;
     int rc = make_range(plan, qm_begin, qm_end, br_begin, br_end, kv_begin, kv_end, parts, &r);
     if (rc != BA_OK) return rc;
@@ -128,8 +129,12 @@ extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main,
             (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
             return rc;
     }
-    if (!(stages & (BA_STAGE_DQ | BA_STAGE_DKDV))) return BA_OK;
+    if (!(stages & (BA_STAGE_DQ | BA_STAGE_DKDV | BA_STAGE_FUSED))) return BA_OK;
     const void *qm = has_main_q ? q_main : nullptr;
+    if (stages & BA_STAGE_FUSED) {
+        if (plan->impl != BA_IMPL_TC || !accumulate) return BA_EUNSUPPORTED;
+        return ba_tc_bwd_fused(plan, r, qm, q_branch, k, v, delta, dO, accumulate, dQ_main, dQ_branch, dK, dV, st);
+    }
     if (plan->impl == BA_IMPL_TC)
         return ba_tc_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK,
                          dV, st, stages);

@@ -232,6 +232,44 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t
     return d;
 }
 
+// The same descriptor as two 32-bit words.  Only the low word holds the address
+// (bits 0-13, in 16-byte units), so the issuing thread keeps one low word per
+// operand and advances it with a 32-bit add per MMA instead of rebuilding the
+// descriptor: one thread issues every MMA of a CTA, and with rebuilt descriptors
+// that thread, not the tensor core, set the pace (about 81 instead of 64 clocks
+// per 128x128x16 MMA).  Shared memory is < 256 KB, so the add cannot carry out
+// of the address field.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+    return ((smem_addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+// high word for 128-byte swizzle, sbo = 1024 bytes
+constexpr uint32_t kSmemDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+// low-word step of a K-major operand tile (two 64-element halves of 16 KB, 32 bytes per K step of 16)
+__host__ __device__ constexpr uint32_t desc_step_kmajor(int ks) { return (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2); }
+// low-word step of an MN-major operand tile (16 rows of 128 bytes per K step)
+__host__ __device__ constexpr uint32_t desc_step_mnmajor(int ks) { return (uint32_t)(ks * 128); }
+
+// D[tmem] (+)= A[smem] * B[smem], descriptors given as (low, high) words
+__device__ __forceinline__ void mma_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %5, 0;\n"
+        "mov.b64 da, {%1, %3};\nmov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kSmemDescHi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %5, 0;\n"
+        "mov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kSmemDescHi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // Instruction descriptor: bf16 x bf16 -> fp32, M x N tile, A K-major,
 // B K-major (b_mn_major = 0) or MN-major (1).
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n, int b_mn_major) {

@@ -12,26 +12,11 @@
 // the same TMEM columns then receive dP, the warps form dS (bf16, written over
 // those columns) and the tensor core adds dS K into the dQ accumulator.
 //   TMEM: R_0 [0,128) R_1 [128,256) (S, then dP, then dS)  dQ_0 [256,384) dQ_1 [384,512)
-#include <limits.h>
-#include <string.h>
-
-#include "ba_common.cuh"
-#include "ba_sm100.cuh"
+#include "ba_tc_bwd.cuh"
 
 using namespace sm100;
 
 namespace {
-
-constexpr int kTile = 128;
-constexpr uint32_t kTileBytes = 32768;
-constexpr float kLog2e = 1.4426950408889634f;
-
-__device__ __forceinline__ uint64_t bit_range(int lo, int hi) {
-    lo = max(lo, 0);
-    hi = min(hi, 63);
-    if (lo > hi) return 0ull;
-    return (~0ull >> (63 - hi)) & (~0ull << lo);
-}
 
 // ============================================================================
 // dQ
@@ -50,48 +35,6 @@ struct DqSmem {
     int abort_flag;
     int lo_min, hi_max, lo_max, hi_min, bs_min, be_max;
 };
-
-struct TcBwdParams {
-    BaMeta meta;
-    BaRange r;
-    const float *nlse2_t, *delta_t;   // head-major [h_q, row_pitch]: -LSE log2(e), delta
-    int64_t row_pitch;
-    void *dq_main, *dq_branch, *dk, *dv;
-    int h_q, h_kv, group, pairs_per_group;
-    float scale, scale_log2;
-    int accumulate;
-    int has_main_q;
-    int main_tiles, total_tiles;      // dQ kernel: query row tiles
-    int main_key_tiles, total_key_tiles;  // dK/dV kernel: key tiles
-    int *status;
-};
-
-template <bool ACC_F32>
-__device__ __forceinline__ void store_grad_chunk(void *dst, size_t elem_off, const uint32_t (&r)[32], float mul) {
-    if (ACC_F32) {
-        float4 *d4 = reinterpret_cast<float4 *>((float *)dst + elem_off);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float4 old = d4[i];
-            old.x += __uint_as_float(r[4 * i]) * mul;
-            old.y += __uint_as_float(r[4 * i + 1]) * mul;
-            old.z += __uint_as_float(r[4 * i + 2]) * mul;
-            old.w += __uint_as_float(r[4 * i + 3]) * mul;
-            d4[i] = old;
-        }
-    } else {
-        uint4 *d4 = reinterpret_cast<uint4 *>((__nv_bfloat16 *)dst + elem_off);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            uint4 v;
-            v.x = pack_bf16(__uint_as_float(r[8 * i]) * mul, __uint_as_float(r[8 * i + 1]) * mul);
-            v.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * mul, __uint_as_float(r[8 * i + 3]) * mul);
-            v.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * mul, __uint_as_float(r[8 * i + 5]) * mul);
-            v.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * mul, __uint_as_float(r[8 * i + 7]) * mul);
-            d4[i] = v;
-        }
-    }
-}
 
 // P = 2^(s * sl2 + neg_lse2) for one 32-column chunk, as 16 packed bf16 pairs
 template <bool MASKED>
@@ -262,38 +205,38 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
         if (lane == 0 && T > 0) {
             constexpr uint32_t IDESC_KMAJ = idesc_bf16(128, 128, 0);  // S = Q K^T, dP = dO V^T
             constexpr uint32_t IDESC_MN = idesc_bf16(128, 128, 1);    // dQ += dS K
-            const uint32_t q_addr[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
-            const uint32_t go_addr[2] = {smem_u32(sm.go[0]), smem_u32(sm.go[1])};
-            auto issue_kmajor = [&](uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-                    mma_ss(d_tmem, smem_desc_sw128(a_addr + off, 16, 1024), smem_desc_sw128(b_addr + off, 16, 1024),
-                           IDESC_KMAJ, ks > 0);
-                }
-            };
-            auto issue_dq = [&](int i, uint32_t k_addr, bool accumulate) {
+            // low descriptor words (the issuing thread advances them with one add per MMA)
+            const uint32_t q_addr[2] = {smem_desc_lo(smem_u32(sm.q[0]), 16), smem_desc_lo(smem_u32(sm.q[1]), 16)};
+            const uint32_t go_addr[2] = {smem_desc_lo(smem_u32(sm.go[0]), 16), smem_desc_lo(smem_u32(sm.go[1]), 16)};
+            const uint32_t k_km[2] = {smem_desc_lo(smem_u32(sm.kbuf[0]), 16), smem_desc_lo(smem_u32(sm.kbuf[1]), 16)};
+            const uint32_t k_mn[2] = {smem_desc_lo(smem_u32(sm.kbuf[0]), 16384), smem_desc_lo(smem_u32(sm.kbuf[1]), 16384)};
+            const uint32_t v_km = smem_desc_lo(smem_u32(sm.vbuf), 16);
+            auto issue_kmajor = [&](uint32_t d_tmem, uint32_t a_km, uint32_t b_km) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + 256 + i * 128, tmem + i * 128 + ks * 8,
-                           smem_desc_sw128(k_addr + ks * 2048, 16384, 1024), IDESC_MN, accumulate || ks > 0);
+                    mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + desc_step_kmajor(ks), IDESC_KMAJ, ks > 0);
+            };
+            auto issue_dq = [&](int i, uint32_t kmn, bool accumulate) {
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, kmn + desc_step_mnmajor(ks), IDESC_MN,
+                              accumulate || ks > 0);
             };
             bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
             ok = ok && mbar_wait(&sm.k_full[0], 0, abort_flag);
             if (ok) {
                 tc_fence_after();
-                issue_kmajor(tmem + 0, q_addr[0], smem_u32(sm.kbuf[0])); tc_commit(&sm.s_full[0]);
-                issue_kmajor(tmem + 128, q_addr[1], smem_u32(sm.kbuf[0])); tc_commit(&sm.s_full[1]);
+                issue_kmajor(tmem + 0, q_addr[0], k_km[0]); tc_commit(&sm.s_full[0]);
+                issue_kmajor(tmem + 128, q_addr[1], k_km[0]); tc_commit(&sm.s_full[1]);
             }
             for (int j = 0; j < T && ok; ++j) {
                 const int kb = j & 1;
-                const uint32_t k_addr = smem_u32(sm.kbuf[kb]);
                 for (int i = 0; i < 2 && ok; ++i) {
                     ok = mbar_wait(&sm.a_done[i], j & 1, abort_flag);
                     if (ok && i == 0) ok = mbar_wait(&sm.v_full, j & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_kmajor(tmem + i * 128, go_addr[i], smem_u32(sm.vbuf));
+                    issue_kmajor(tmem + i * 128, go_addr[i], v_km);
                     tc_commit(&sm.dp_full[i]);
                     if (i == 1) tc_commit(&sm.v_empty);
                 }
@@ -301,7 +244,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
                     ok = mbar_wait(&sm.b_done[i], j & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_dq(i, k_addr, j > 0);
+                    issue_dq(i, k_mn[kb], j > 0);
                     if (i == 1) tc_commit(&sm.k_empty[kb]);
                     if (j + 1 < T) {
                         if (i == 0) {
@@ -309,7 +252,7 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
                             if (!ok) break;
                             tc_fence_after();
                         }
-                        issue_kmajor(tmem + i * 128, q_addr[i], smem_u32(sm.kbuf[kb ^ 1]));
+                        issue_kmajor(tmem + i * 128, q_addr[i], k_km[kb ^ 1]);
                         tc_commit(&sm.s_full[i]);
                     } else {
                         tc_commit(&sm.dq_full[i]);
@@ -691,18 +634,21 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
         if (lane == 0 && n_iter > 0) {
             constexpr uint32_t IDESC_T = idesc_bf16(128, kSub, 0);   // 128 keys x 64 rows, K = d
             constexpr uint32_t IDESC_ACC = idesc_bf16(128, 128, 1);  // 128 keys x 128 d, K = 64 rows
-            const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v);
-            auto issue_t = [&](uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+            // low descriptor words (the issuing thread advances them with one add per MMA);
+            // a stage holds the Q sub-tile, then the dO sub-tile, each two 64-column halves of 8 KB
+            const uint32_t k_km = smem_desc_lo(smem_u32(sm.k), 16), v_km = smem_desc_lo(smem_u32(sm.v), 16);
+            const uint32_t qs_km0 = smem_desc_lo(smem_u32(sm.qs[0]), 16), qs_mn0 = smem_desc_lo(smem_u32(sm.qs[0]), 8192);
+            constexpr uint32_t kStageStep = (2 * kSubBytes) >> 4, kHalfStage = kSubBytes >> 4;
+            auto issue_t = [&](uint32_t d_tmem, uint32_t a_km, uint32_t b_km) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ss(d_tmem, smem_desc_sw128(a_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                           smem_desc_sw128(b_addr + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), IDESC_T, ks > 0);
+                    mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + (uint32_t)((ks >> 2) * 512 + (ks & 3) * 2),
+                              IDESC_T, ks > 0);
             };
-            auto issue_acc = [&](uint32_t d_tmem, uint32_t a_tmem, uint32_t b_addr, bool accumulate) {
+            auto issue_acc = [&](uint32_t d_tmem, uint32_t a_tmem, uint32_t b_mn, bool accumulate) {
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    mma_ts(d_tmem, a_tmem + ks * 8, smem_desc_sw128(b_addr + ks * 2048, 8192, 1024), IDESC_ACC,
-                           accumulate || ks > 0);
+                    mma_ts_lh(d_tmem, a_tmem + ks * 8, b_mn + desc_step_mnmajor(ks), IDESC_ACC, accumulate || ks > 0);
             };
             bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
             for (int b = 0; b < 2 && ok; ++b) {
@@ -710,27 +656,27 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
                 ok = mbar_wait(&sm.q_full[b], 0, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_t(tmem + 256 + b * 128, k_addr, smem_u32(sm.qs[b]));                    // S^T = K Q^T
-                issue_t(tmem + 256 + b * 128 + 64, v_addr, smem_u32(sm.qs[b]) + kSubBytes);   // dP^T = V dO^T
+                issue_t(tmem + 256 + b * 128, k_km, qs_km0 + b * kStageStep);                    // S^T = K Q^T
+                issue_t(tmem + 256 + b * 128 + 64, v_km, qs_km0 + b * kStageStep + kHalfStage);  // dP^T = V dO^T
                 tc_commit(&sm.sd_full[b]);
             }
             for (int t = 0; t < n_iter && ok; ++t) {
                 const int b = t & 1;
-                const uint32_t stage_addr = smem_u32(sm.qs[t % kQStages]);
+                const uint32_t stage_mn = qs_mn0 + (t % kQStages) * kStageStep;
                 ok = mbar_wait(&sm.pd_done[b], (t >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_acc(tmem + 128, tmem + 256 + b * 128, stage_addr + kSubBytes, t > 0);   // dV += P^T dO
-                issue_acc(tmem + 0, tmem + 256 + b * 128 + 64, stage_addr, t > 0);             // dK += dS^T Q
+                issue_acc(tmem + 128, tmem + 256 + b * 128, stage_mn + kHalfStage, t > 0);   // dV += P^T dO
+                issue_acc(tmem + 0, tmem + 256 + b * 128 + 64, stage_mn, t > 0);             // dK += dS^T Q
                 tc_commit(&sm.q_empty[t % kQStages]);
                 const int t2 = t + 2;
                 if (t2 < n_iter) {
-                    const uint32_t next_addr = smem_u32(sm.qs[t2 % kQStages]);
+                    const uint32_t next_km = qs_km0 + (t2 % kQStages) * kStageStep;
                     ok = mbar_wait(&sm.q_full[t2 % kQStages], (t2 / kQStages) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_t(tmem + 256 + b * 128, k_addr, next_addr);
-                    issue_t(tmem + 256 + b * 128 + 64, v_addr, next_addr + kSubBytes);
+                    issue_t(tmem + 256 + b * 128, k_km, next_km);
+                    issue_t(tmem + 256 + b * 128 + 64, v_km, next_km + kHalfStage);
                     tc_commit(&sm.sd_full[b]);
                 }
             }

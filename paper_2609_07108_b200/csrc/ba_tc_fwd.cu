@@ -261,22 +261,22 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
         if (lane == 0 && T > 0) {
             constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, 0);
             constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, 1);
-            const uint32_t q_addr[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
+            // low descriptor words (the issuing thread advances them with one add per MMA)
+            const uint32_t q_km[2] = {smem_desc_lo(smem_u32(sm.q[0]), 16), smem_desc_lo(smem_u32(sm.q[1]), 16)};
+            const uint32_t kv_km0 = smem_desc_lo(smem_u32(sm.kv[0]), 16), kv_mn0 = smem_desc_lo(smem_u32(sm.kv[0]), 16384);
+            constexpr uint32_t kStageStep = kTileBytes >> 4;
             auto issue_qk = [&](int i, int stage) {
-                const uint32_t k_addr = smem_u32(sm.kv[stage]);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-                    mma_ss(tmem + i * 128, smem_desc_sw128(q_addr[i] + off, 16, 1024),
-                           smem_desc_sw128(k_addr + off, 16, 1024), IDESC_QK, ks > 0);
-                }
-            };
-            auto issue_pv = [&](int i, int stage, bool accumulate) {
-                const uint32_t v_addr = smem_u32(sm.kv[stage]);
+                const uint32_t k_km = kv_km0 + stage * kStageStep;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + 256 + i * 128, tmem + i * 128 + ks * 8,
-                           smem_desc_sw128(v_addr + ks * 2048, 16384, 1024), IDESC_PV, accumulate || ks > 0);
+                    mma_ss_lh(tmem + i * 128, q_km[i] + desc_step_kmajor(ks), k_km + desc_step_kmajor(ks), IDESC_QK, ks > 0);
+            };
+            auto issue_pv = [&](int i, int stage, bool accumulate) {
+                const uint32_t v_mn = kv_mn0 + stage * kStageStep;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, v_mn + desc_step_mnmajor(ks), IDESC_PV,
+                              accumulate || ks > 0);
             };
             bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
             ok = ok && mbar_wait(&sm.kv_full[0], 0, abort_flag);

@@ -141,10 +141,11 @@ def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None):
     return out, lse, launches
 
 
-def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp):
+def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp, fused=False):
     """Emulated CP backward: the same (rank, step) blocks, gradients accumulated
     in fp32 and converted once at the end.  Returns (dQ_main, dQ_branch, dK, dV,
-    launches) in the input dtype."""
+    launches) in the input dtype.  `fused`: one kernel per block for dQ, dK and
+    dV (dQ summed with atomic adds) instead of a dQ and a dK/dV kernel."""
     import torch
     p = plan.problem
     f32 = dict(dtype=torch.float32, device=plan.device)
@@ -156,7 +157,8 @@ def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp):
     for b in schedule(p, cp):
         parts = ba.PART_MAIN | (ba.PART_BRANCH if b.branch_part else 0)
         ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=b.qm, br_range=b.br,
-                           kv_range=b.kv, parts=parts, accumulate=True, grads=grads)
-        launches += 4
+                           kv_range=b.kv, parts=parts, accumulate=True, grads=grads,
+                           stages=ba.STAGE_ALL_FUSED if fused else ba.STAGE_ALL)
+        launches += 3 if fused else 4
     outs = tuple(ba.ba_finalize_grads(g, dtype=plan.torch_dtype) for g in grads)
     return (*outs, launches + 4)
