@@ -586,7 +586,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="auto", choices=["auto", *WORKLOADS])
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tc"])
-    ap.add_argument("--bwd", default="split", choices=["split", "fused"],
+    ap.add_argument("--bwd", default="fused", choices=["split", "fused"],
                     help="backward of the chunked workloads: dQ kernel + dK/dV kernel, or one kernel "
                          "for all three (dQ summed with atomic adds)")
     ap.add_argument("--branch-only", action="store_true",
