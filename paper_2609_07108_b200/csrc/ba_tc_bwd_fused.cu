@@ -23,8 +23,9 @@
 //
 // Warps 0-3 / 4-7 work on query columns [0,64) / [64,128) of every tile: A(t) P^T
 // from S^T, then B(t) dS^T from dP^T.  Warps 8-11 read dQ^T out of X (R(t)) and
-// issue the reductions, warp 12 issues the MMAs, warp 13 runs the copies:
-//   MMA:    dV(t)  dP(t) [after R(t-1)]  S(t+1)  dQ(t) dK(t) [after B(t)]
+// issue the reductions, warp 13 runs the copies, one thread each of warps 12 and 14
+// issues MMAs:  warp 12: dP(t) [after R(t-1)], dQ(t) dK(t) [after B(t)]
+//               warp 14: dV(t) [after A(t)], S(t+1)
 // The warpgroups re-split the register file (setmaxnreg) for their roles.
 #include "ba_tc_bwd.cuh"
 
@@ -152,7 +153,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
 
     if (tid == 0) {
         mbar_init(&sm.kv_full, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sm.q_full[s], 1); mbar_init(&sm.q_empty[s], 2); }
         mbar_init(&sm.s_full, 1);
         mbar_init(&sm.a_done, 256);
         mbar_init(&sm.dp_full, 1);
@@ -160,7 +161,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
         mbar_init(&sm.dq_full, 1);
         mbar_init(&sm.r_done, 128);
         mbar_init(&sm.dk_done, 1);
-        mbar_init(&sm.acc_full, 1);
+        mbar_init(&sm.acc_full, 2);
         sm.abort_flag = 0;
         sm.qend_max = -1; sm.bq0_min = INT_MAX; sm.bq1_max = -1;
         fence_barrier_init();
@@ -284,8 +285,16 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                 while (!mbar_try_wait(&sm.kv_full, 0) && ++spins < (1u << 22)) {}
             }
         }
-      } else if (warp == 12) {
-        // ================================================= MMA issuer
+      } else if (warp == 12 || warp == 14) {
+        // ================================================= MMA issuers
+        // Two issuing threads with independent streams, because one thread cannot feed the
+        // tensor core here: a tcgen05.mma costs its thread about 53 clocks on an idle SM (a
+        // 128x128x16 MMA runs 64) and several times that while the other warps of its
+        // scheduler are busy.
+        //   warp 12: dP^T(t) [after R(t-1)], dQ^T(t) and dK(t) [after B(t)]   -- X, dK
+        //   warp 14: dV(t) [after A(t)], S^T(t+1)                             -- S^T / P^T, dV
+        // No order is needed between the two streams; each keeps its own order by issuing
+        // from one thread.  A Q / dO stage is released by both (q_empty counts 2).
         if (lane == 0 && n_iter > 0) {
             constexpr uint32_t IDESC_T = idesc_bf16_full(128, 128, 0, 0);    // S^T, dP^T: both operands K-major
             constexpr uint32_t IDESC_ACC = idesc_bf16_full(128, 128, 0, 1);  // dV, dK: B = dO / Q rows, MN-major
@@ -306,53 +315,64 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
             };
             bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
             ok = ok && mbar_wait(&sm.q_full[0], 0, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                issue_t(t_s, k_km, q_km0);   tc_commit(&sm.s_full);    // S^T(0)
-                issue_t(t_x, v_km, go_km0);  tc_commit(&sm.dp_full);   // dP^T(0)
-            }
-            for (int t = 0; t < n_iter && ok; ++t) {
-                const int st = t & 1;
-                const uint32_t q_mn = q_mn0 + st * kStageStep, go_km = go_km0 + st * kStageStep;
-                const uint32_t go_mn = go_mn0 + st * kStageStep, q_km_next = q_km0 + (st ^ 1) * kStageStep;
-                // --- dV += P^T dO  (P^T: bf16 pairs in columns [0,32) and [64,96) of the S^T region)
-                ok = mbar_wait(&sm.a_done, t & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts_lh(t_dv, t_s + (ks >> 2) * 64 + (ks & 3) * 8, go_mn + desc_step_mnmajor(ks), IDESC_ACC,
-                              t > 0 || ks > 0);
-                // --- dP^T(t) into X once dQ^T(t-1) has been read out of it
-                if (t > 0) {
-                    ok = mbar_wait(&sm.r_done, (t - 1) & 1, abort_flag);
+            if (warp == 12) {
+                if (ok) {
+                    tc_fence_after();
+                    issue_t(t_x, v_km, go_km0);  tc_commit(&sm.dp_full);   // dP^T(0)
+                }
+                for (int t = 0; t < n_iter && ok; ++t) {
+                    const int st = t & 1;
+                    const uint32_t q_mn = q_mn0 + st * kStageStep, go_km = go_km0 + st * kStageStep;
+                    // --- dP^T(t) into X once dQ^T(t-1) has been read out of it
+                    if (t > 0) {
+                        ok = mbar_wait(&sm.r_done, (t - 1) & 1, abort_flag);
+                        if (ok) ok = mbar_wait(&sm.q_full[st], (t >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_t(t_x, v_km, go_km);
+                        tc_commit(&sm.dp_full);
+                    }
+                    // --- dQ^T(t) = K_j^T dS^T into X, dK += dS^T Q
+                    ok = mbar_wait(&sm.b_done, t & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_t(t_x, v_km, go_km);
-                    tc_commit(&sm.dp_full);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ss_lh(t_x, k_mn + desc_step_mnmajor(ks), ds_mn + desc_step_mnmajor(ks), IDESC_DQ, ks > 0);
+                    tc_commit(&sm.dq_full);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ss_lh(t_dk, ds_km + desc_step_kmajor(ks), q_mn + desc_step_mnmajor(ks), IDESC_ACC,
+                                  t > 0 || ks > 0);
+                    tc_commit(&sm.dk_done);
+                    tc_commit(&sm.q_empty[st]);
                 }
-                // --- S^T(t+1): P^T(t) is consumed by the dV MMAs queued above
-                if (t + 1 < n_iter) {
-                    ok = mbar_wait(&sm.q_full[st ^ 1], ((t + 1) >> 1) & 1, abort_flag);
+            } else {
+                if (ok) {
+                    tc_fence_after();
+                    issue_t(t_s, k_km, q_km0);   tc_commit(&sm.s_full);    // S^T(0)
+                }
+                for (int t = 0; t < n_iter && ok; ++t) {
+                    const int st = t & 1;
+                    const uint32_t go_mn = go_mn0 + st * kStageStep, q_km_next = q_km0 + (st ^ 1) * kStageStep;
+                    // --- dV += P^T dO  (P^T: bf16 pairs in columns [0,32) and [64,96) of the S^T region)
+                    ok = mbar_wait(&sm.a_done, t & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_t(t_s, k_km, q_km_next);
-                    tc_commit(&sm.s_full);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ts_lh(t_dv, t_s + (ks >> 2) * 64 + (ks & 3) * 8, go_mn + desc_step_mnmajor(ks), IDESC_ACC,
+                                  t > 0 || ks > 0);
+                    tc_commit(&sm.q_empty[st]);
+                    // --- S^T(t+1): P^T(t) is consumed by the dV MMAs queued above
+                    if (t + 1 < n_iter) {
+                        ok = mbar_wait(&sm.q_full[st ^ 1], ((t + 1) >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_t(t_s, k_km, q_km_next);
+                        tc_commit(&sm.s_full);
+                    }
                 }
-                // --- dQ^T(t) = K_j^T dS^T into X, dK += dS^T Q
-                ok = mbar_wait(&sm.b_done, t & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ss_lh(t_x, k_mn + desc_step_mnmajor(ks), ds_mn + desc_step_mnmajor(ks), IDESC_DQ, ks > 0);
-                tc_commit(&sm.dq_full);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ss_lh(t_dk, ds_km + desc_step_kmajor(ks), q_mn + desc_step_mnmajor(ks), IDESC_ACC,
-                              t > 0 || ks > 0);
-                tc_commit(&sm.dk_done);
-                tc_commit(&sm.q_empty[st]);
             }
             if (ok) tc_commit(&sm.acc_full);
         }
