@@ -295,7 +295,10 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
         //   warp 14: dV(t) [after A(t)], S^T(t+1)                             -- S^T / P^T, dV
         // No order is needed between the two streams; each keeps its own order by issuing
         // from one thread.  A Q / dO stage is released by both (q_empty counts 2).
-        if (lane == 0 && n_iter > 0) {
+        // The whole warp runs the code and an elected lane issues each MMA and commit: with
+        // warp-uniform control flow the descriptors stay in uniform registers, which halves
+        // the cost of a tcgen05.mma for its thread.
+        if (n_iter > 0) {
             constexpr uint32_t IDESC_T = idesc_bf16_full(128, 128, 0, 0);    // S^T, dP^T: both operands K-major
             constexpr uint32_t IDESC_ACC = idesc_bf16_full(128, 128, 0, 1);  // dV, dK: B = dO / Q rows, MN-major
             constexpr uint32_t IDESC_DQ = idesc_bf16_full(128, 128, 1, 1);   // dQ^T: A = K_j rows, B = dS^T rows
@@ -311,70 +314,74 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
             auto issue_t = [&](uint32_t d_tmem, uint32_t a_km, uint32_t b_km) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + desc_step_kmajor(ks), IDESC_T, ks > 0);
+                    if (elect_one()) mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + desc_step_kmajor(ks), IDESC_T, ks > 0);
             };
-            bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
-            ok = ok && mbar_wait(&sm.q_full[0], 0, abort_flag);
+            // every lane waits (and all agree on the outcome, so the warp stays converged)
+            auto wait = [&](uint64_t *bar, uint32_t parity) {
+                return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+            };
+            bool ok = wait(&sm.kv_full, 0);
+            ok = ok && wait(&sm.q_full[0], 0);
             if (warp == 12) {
                 if (ok) {
                     tc_fence_after();
-                    issue_t(t_x, v_km, go_km0);  tc_commit(&sm.dp_full);   // dP^T(0)
+                    issue_t(t_x, v_km, go_km0);  if (elect_one()) tc_commit(&sm.dp_full);   // dP^T(0)
                 }
                 for (int t = 0; t < n_iter && ok; ++t) {
                     const int st = t & 1;
                     const uint32_t q_mn = q_mn0 + st * kStageStep, go_km = go_km0 + st * kStageStep;
                     // --- dP^T(t) into X once dQ^T(t-1) has been read out of it
                     if (t > 0) {
-                        ok = mbar_wait(&sm.r_done, (t - 1) & 1, abort_flag);
-                        if (ok) ok = mbar_wait(&sm.q_full[st], (t >> 1) & 1, abort_flag);
+                        ok = wait(&sm.r_done, (t - 1) & 1);
+                        if (ok) ok = wait(&sm.q_full[st], (t >> 1) & 1);
                         if (!ok) break;
                         tc_fence_after();
                         issue_t(t_x, v_km, go_km);
-                        tc_commit(&sm.dp_full);
+                        if (elect_one()) tc_commit(&sm.dp_full);
                     }
                     // --- dQ^T(t) = K_j^T dS^T into X, dK += dS^T Q
-                    ok = mbar_wait(&sm.b_done, t & 1, abort_flag);
+                    ok = wait(&sm.b_done, t & 1);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        mma_ss_lh(t_x, k_mn + desc_step_mnmajor(ks), ds_mn + desc_step_mnmajor(ks), IDESC_DQ, ks > 0);
-                    tc_commit(&sm.dq_full);
+                        if (elect_one()) mma_ss_lh(t_x, k_mn + desc_step_mnmajor(ks), ds_mn + desc_step_mnmajor(ks), IDESC_DQ, ks > 0);
+                    if (elect_one()) tc_commit(&sm.dq_full);
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        mma_ss_lh(t_dk, ds_km + desc_step_kmajor(ks), q_mn + desc_step_mnmajor(ks), IDESC_ACC,
+                        if (elect_one()) mma_ss_lh(t_dk, ds_km + desc_step_kmajor(ks), q_mn + desc_step_mnmajor(ks), IDESC_ACC,
                                   t > 0 || ks > 0);
-                    tc_commit(&sm.dk_done);
-                    tc_commit(&sm.q_empty[st]);
+                    if (elect_one()) tc_commit(&sm.dk_done);
+                    if (elect_one()) tc_commit(&sm.q_empty[st]);
                 }
             } else {
                 if (ok) {
                     tc_fence_after();
-                    issue_t(t_s, k_km, q_km0);   tc_commit(&sm.s_full);    // S^T(0)
+                    issue_t(t_s, k_km, q_km0);   if (elect_one()) tc_commit(&sm.s_full);    // S^T(0)
                 }
                 for (int t = 0; t < n_iter && ok; ++t) {
                     const int st = t & 1;
                     const uint32_t go_mn = go_mn0 + st * kStageStep, q_km_next = q_km0 + (st ^ 1) * kStageStep;
                     // --- dV += P^T dO  (P^T: bf16 pairs in columns [0,32) and [64,96) of the S^T region)
-                    ok = mbar_wait(&sm.a_done, t & 1, abort_flag);
+                    ok = wait(&sm.a_done, t & 1);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        mma_ts_lh(t_dv, t_s + (ks >> 2) * 64 + (ks & 3) * 8, go_mn + desc_step_mnmajor(ks), IDESC_ACC,
+                        if (elect_one()) mma_ts_lh(t_dv, t_s + (ks >> 2) * 64 + (ks & 3) * 8, go_mn + desc_step_mnmajor(ks), IDESC_ACC,
                                   t > 0 || ks > 0);
-                    tc_commit(&sm.q_empty[st]);
+                    if (elect_one()) tc_commit(&sm.q_empty[st]);
                     // --- S^T(t+1): P^T(t) is consumed by the dV MMAs queued above
                     if (t + 1 < n_iter) {
-                        ok = mbar_wait(&sm.q_full[st ^ 1], ((t + 1) >> 1) & 1, abort_flag);
+                        ok = wait(&sm.q_full[st ^ 1], ((t + 1) >> 1) & 1);
                         if (!ok) break;
                         tc_fence_after();
                         issue_t(t_s, k_km, q_km_next);
-                        tc_commit(&sm.s_full);
+                        if (elect_one()) tc_commit(&sm.s_full);
                     }
                 }
             }
-            if (ok) tc_commit(&sm.acc_full);
+            if (ok) if (elect_one()) tc_commit(&sm.acc_full);
         }
       }
     } else if (warp >= 8) {
