@@ -94,10 +94,12 @@ __device__ __forceinline__ void chunk_dst(const uint32_t (&r)[32], const uint32_
         const uint32_t pa = pr[e >> 1], pb = pr[(e >> 1) + 1];
         const float2 fa = make_float2(__uint_as_float(pa << 16), __uint_as_float(pa & 0xffff0000u));
         const float2 fb = make_float2(__uint_as_float(pb << 16), __uint_as_float(pb & 0xffff0000u));
-        float2 d0 = fmul2(fa, fadd2(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])),
-                                    make_float2(-dv.x, -dv.y)));
-        float2 d1 = fmul2(fb, fadd2(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])),
-                                    make_float2(-dv.z, -dv.w)));
+        // dP - delta as one packed fma (delta * -1 + dP): no separate negations
+        const float2 m1 = make_float2(-1.f, -1.f);
+        float2 d0 = fmul2(fa, ffma2(make_float2(dv.x, dv.y), m1,
+                                    make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1]))));
+        float2 d1 = fmul2(fb, ffma2(make_float2(dv.z, dv.w), m1,
+                                    make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]))));
         if (MASKED) {
             d0.x = ((mk >> e) & 1u) ? d0.x : 0.f;
             d0.y = ((mk >> (e + 1)) & 1u) ? d0.y : 0.f;
