@@ -69,7 +69,7 @@ def visible_counts(p):
     return np.concatenate([main, np.repeat(prefix, blen) + local])
 
 
-def check_sampled(ba, oracle, p, cp, groups, n_rows, seed, backward=True, edges=()):
+def check_sampled(ba, oracle, p, cp, groups, n_rows, seed, backward=True, edges=(), fused=False):
     plan = ba.Plan(p, impl=ba.IMPL_TC)
     assert plan.impl == ba.IMPL_TC
     t = device_inputs(p, seed)
@@ -106,7 +106,8 @@ def check_sampled(ba, oracle, p, cp, groups, n_rows, seed, backward=True, edges=
         d_o = torch.zeros_like(t["d_o"])
         d_o[rows_t] = t["d_o"][rows_t]
         if cp:
-            dqm, dqb, dk, dv, _ = zigzag.backward(ba, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, d_o, cp)
+            dqm, dqb, dk, dv, _ = zigzag.backward(ba, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, d_o, cp,
+                                                  fused=fused)
         else:
             dqm, dqb, dk, dv = ba.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, d_o)
         plan.check()
@@ -157,18 +158,21 @@ def test_config4_full_size(ba, oracle):
     check_sampled(ba, oracle, p, cp=0, groups=[2, 5], n_rows=512, seed=2, edges=tile_edges(p))
 
 
-def test_config5_full_size_zigzag(ba, oracle):
+@pytest.mark.parametrize("fused", [False, True], ids=["split_bwd", "fused_bwd"])
+def test_config5_full_size_zigzag(ba, oracle, fused):
     """256K tokens through the emulated 8-way zigzag layout: partial forward +
-    lse_merge, partial backward with fp32 accumulation."""
+    lse_merge, partial backward with fp32 accumulation (dQ kernel + dK/dV kernel, or
+    the one-kernel backward that bench.py times)."""
     p = W.config5()
     chunk = p.n_main // 16
     edges = [0, 1, p.n_main - 1]
     for c in range(16):
         edges += [c * chunk, (c + 1) * chunk - 1]
-    check_sampled(ba, oracle, p, cp=8, groups=[3], n_rows=160, seed=3, edges=edges)
+    check_sampled(ba, oracle, p, cp=8, groups=[3], n_rows=160, seed=3, edges=edges, fused=fused)
 
 
-def test_zigzag_equals_monolithic_small(ba):
+@pytest.mark.parametrize("fused", [False, True], ids=["split_bwd", "fused_bwd"])
+def test_zigzag_equals_monolithic_small(ba, fused):
     """Self-consistency of the two launch configurations on the GPU."""
     p = W.config5(shrink=16)
     plan = ba.Plan(p, impl=ba.IMPL_TC)
@@ -178,7 +182,7 @@ def test_zigzag_equals_monolithic_small(ba):
     assert float((o1.float() - o2.float()).abs().max()) <= 2e-2
     assert float((l1 - l2).abs().max()) <= 1e-3
     g1 = ba.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o1, l1, t["d_o"])
-    g2 = zigzag.backward(ba, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o1, l1, t["d_o"], 8)
+    g2 = zigzag.backward(ba, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o1, l1, t["d_o"], 8, fused=fused)
     for a, b in zip(g1, g2[:4]):
         assert float((a.float() - b.float()).abs().max()) <= 2e-2
     plan.check()
@@ -205,10 +209,20 @@ def test_config3_full_size_dense_cotangent_one_group(ba, oracle):
     assert_close("dQ", f32(torch.cat([dqm, dqb], 0)[:, qh_t]), ref_dq, tol)
     assert_close("dK", f32(dk[:, 4:5]), ref_dk, tol)
     assert_close("dV", f32(dv[:, 4:5]), ref_dv, tol)
+    # the one-kernel backward on the same dense cotangent (fp32 accumulators, dQ by atomic adds)
+    del dqm, dqb, dk, dv
+    fq, fb, fk, fv = ba.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"],
+                                        accumulate=True, stages=ba.STAGE_ALL_FUSED)
+    plan.check()
+    assert_close("dQ fused", f32(torch.cat([fq, fb], 0)[:, qh_t]), ref_dq, tol)
+    assert_close("dK fused", f32(fk[:, 4:5]), ref_dk, tol)
+    assert_close("dV fused", f32(fv[:, 4:5]), ref_dv, tol)
 
 
 def test_results_are_bit_identical_from_run_to_run(ba):
-    """Every output element has one owning CTA and a fixed summation order."""
+    """Forward and the two-kernel backward: every output element has one owning CTA
+    and a fixed summation order.  (The one-kernel backward sums dQ with atomic adds;
+    its dK / dV are bit-identical, its dQ only close: test_gpu_fused_bwd.py.)"""
     p = W.config4(shrink=8)
     plan = ba.Plan(p, impl=ba.IMPL_TC)
     t = device_inputs(p, 12)
