@@ -198,12 +198,16 @@ class Recorder:
         ba = self.ba
         k = dict(k)
         fused = k.pop("stages", ba.STAGE_ALL) == ba.STAGE_ALL_FUSED
+        # gradients in the input dtype through the one-kernel backward: all stages share the larger workspace
+        prep_kw = {"fused_scratch": True} if fused and not k.get("accumulate", False) else {}
         out = self._wrap("bwd_prep", 2 if q_main is not None else 1, ba.branch_attn_bwd, plan, q_main, *a,
-                         stages=ba.STAGE_PREP, **k)
+                         stages=ba.STAGE_PREP, **prep_kw, **k)
         k2 = dict(k)
         k2["grads"] = out
         if fused:   # one kernel for dQ, dK and dV
-            return self._wrap("bwd_fused", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_FUSED, **k2)
+            # (without accumulate: plus the conversion of the dQ accumulators of main and branch rows)
+            n_l = 1 if k.get("accumulate", False) else (3 if q_main is not None else 2)
+            return self._wrap("bwd_fused", n_l, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_FUSED, **k2)
         self._wrap("bwd_dq", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DQ, **k2)
         return self._wrap("bwd_dkdv", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DKDV, **k2)
 
@@ -245,7 +249,8 @@ def run_step(rec, plan, t, cp, backward, fused=False):
         o, lse = rec.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"],
                                      out=t.get("_o"), lse=t.get("_lse"))
         grads = rec.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"],
-                                    grads=t.get("_grads")) if backward else None
+                                    grads=t.get("_grads"),
+                                    stages=rec.STAGE_ALL_FUSED if fused else rec.STAGE_ALL) if backward else None
     return o, lse, grads
 
 
@@ -287,8 +292,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # the one-kernel backward adds into fp32 accumulators: the chunked (zigzag) path has them
-    fused = args.bwd == "fused" and bool(cp) and plan.impl == ba.IMPL_TC
+    fused = args.bwd == "fused" and plan.impl == ba.IMPL_TC
     for _ in range(args.warmup):
         run_step(rec, plan, t, cp, backward, fused=fused)
         if flush is not None:
@@ -450,7 +454,7 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     for _ in range(steps):
         for k in names:
             h2d_copy(t[k], k)
-        o, lse, grads = run_step(rec, plan, t, cp, backward, fused=args.bwd == "fused" and bool(cp))
+        o, lse, grads = run_step(rec, plan, t, cp, backward, fused=args.bwd == "fused" and plan.impl == ba.IMPL_TC)
         outs = [o, lse] + (list(grads[:4]) if backward else [])
         outs = [x for x in outs if x is not None]
         for i, src in enumerate(outs):
@@ -587,8 +591,8 @@ def main():
     ap.add_argument("--workload", default="auto", choices=["auto", *WORKLOADS])
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--bwd", default="fused", choices=["split", "fused"],
-                    help="backward of the chunked workloads: dQ kernel + dK/dV kernel, or one kernel "
-                         "for all three (dQ summed with atomic adds)")
+                    help="backward: dQ kernel + dK/dV kernel, or one kernel for all three (dQ summed "
+                         "with atomic adds)")
     ap.add_argument("--branch-only", action="store_true",
                     help="q_main = NULL: only the branch tokens are queries (monolithic workloads)")
     ap.add_argument("--no-e2e", action="store_true")

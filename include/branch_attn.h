@@ -49,7 +49,7 @@ typedef enum ba_status {
 enum { BA_BF16 = 0, BA_FP32 = 1 };
 enum { BA_MASK_CHAIN = 0, BA_MASK_BLOCK = 1, BA_MASK_TREE = 2 };
 enum { BA_PART_MAIN = 1, BA_PART_BRANCH = 2 };
-enum { BA_OP_FWD = 0, BA_OP_BWD = 1 };
+enum { BA_OP_FWD = 0, BA_OP_BWD = 1, BA_OP_BWD_FUSED = 2 };
 enum { BA_STAGE_PREP = 1, BA_STAGE_DQ = 2, BA_STAGE_DKDV = 4, BA_STAGE_ALL = 7,
        BA_STAGE_FUSED = 8, BA_STAGE_ALL_FUSED = 9 };
 
@@ -102,7 +102,10 @@ int ba_plan_create(const ba_problem_t *p, void *plan_mem, size_t plan_bytes, voi
                    ba_plan_t **out);
 int ba_plan_destroy(ba_plan_t *plan);
 
-/* Scratch bytes (device, 256-byte aligned) that `op` needs; may be 0. */
+/* Scratch bytes (device, 256-byte aligned) that `op` needs; may be 0.
+ * BA_OP_BWD_FUSED = BA_OP_BWD plus an fp32 dQ accumulator of (N + M) * h_q * head_dim
+ * floats: what BA_STAGE_FUSED needs when the gradients are written in the input
+ * dtype (accumulate = 0). */
 size_t ba_workspace_bytes(const ba_plan_t *plan, int op);
 
 /* Exact number of (query row, visible key) pairs per query head of the whole
@@ -193,9 +196,13 @@ int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const void *q_bra
  *                  with them) by ONE key-stationary kernel that forms S and dP
  *                  once per tile pair (10 D flop per visible pair instead of 14 D)
  *                  and sums dQ into its fp32 accumulator with atomic adds.
- *                  Needs accumulate = 1 and the tensor-core kernels, else
- *                  BA_EUNSUPPORTED.  dK and dV stay bit-reproducible; the last
- *                  bits of dQ depend on the order in which the key tiles arrive.
+ *                  Needs the tensor-core kernels, else BA_EUNSUPPORTED.  With
+ *                  accumulate = 0 the workspace must hold
+ *                  ba_workspace_bytes(plan, BA_OP_BWD_FUSED) (all stages of one
+ *                  backward use the same workspace): dQ is summed there in fp32
+ *                  and converted at the end.  dK and dV stay bit-reproducible;
+ *                  the last bits of dQ depend on the order in which the key
+ *                  tiles arrive.
  *   BA_STAGE_ALL_FUSED = BA_STAGE_PREP | BA_STAGE_FUSED.
  */
 int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main, const void *q_branch,

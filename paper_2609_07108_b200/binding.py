@@ -17,7 +17,7 @@ from . import build as _build
 
 BA_BF16, BA_FP32 = 0, 1
 PART_MAIN, PART_BRANCH, PART_ALL = 1, 2, 3
-OP_FWD, OP_BWD = 0, 1
+OP_FWD, OP_BWD, OP_BWD_FUSED = 0, 1, 2
 STAGE_PREP, STAGE_DQ, STAGE_DKDV, STAGE_ALL = 1, 2, 4, 7
 STAGE_FUSED, STAGE_ALL_FUSED = 8, 9
 IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
@@ -238,9 +238,12 @@ def lse_merge(o_a, lse_a, o_b, lse_b, out=None, lse_out=None, out_dtype=torch.fl
 
 
 def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br_range=None,
-                    kv_range=None, parts=PART_ALL, accumulate=False, grads=None, stages=STAGE_ALL):
+                    kv_range=None, parts=PART_ALL, accumulate=False, grads=None, stages=STAGE_ALL,
+                    fused_scratch=False):
     """(dQ_main, dQ_branch, dK, dV).  With `accumulate`, `grads` must hold four
-    zero-initialised fp32 tensors which receive the selected terms."""
+    zero-initialised fp32 tensors which receive the selected terms.  `fused_scratch`:
+    this call prepares (STAGE_PREP) a backward whose STAGE_FUSED call follows
+    separately with accumulate=False."""
     p = plan.problem
     qm_range = (0, p.n_main) if qm_range is None else qm_range
     br_range = (0, p.num_branches) if br_range is None else br_range
@@ -253,7 +256,12 @@ def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br
                  mk((p.n_branch, p.h_q, p.head_dim), dtype=dt, device=plan.device),
                  mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device),
                  mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device))
-    ws = plan.workspace(OP_BWD)
+    # every stage of one backward must see the same workspace: once a plan has been
+    # used for the one-kernel backward with gradients in the input dtype (which keeps
+    # an fp32 dQ accumulator in the workspace), all its backward calls use that buffer
+    if fused_scratch or ((stages & STAGE_FUSED) and not accumulate):
+        plan._fused_ws = True
+    ws = plan.workspace(OP_BWD_FUSED if getattr(plan, "_fused_ws", False) else OP_BWD)
     args = (plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(o), _p(lse),
             _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1],
             kv_range[0], kv_range[1], parts, 1 if accumulate else 0,

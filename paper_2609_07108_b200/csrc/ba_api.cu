@@ -39,8 +39,12 @@ int make_range(const ba_plan *pl, int64_t qm_begin, int64_t qm_end, int64_t br_b
 
 extern "C" size_t ba_workspace_bytes(const ba_plan_t *plan, int op) {
     if (!plan) return 0;
-    if (op == BA_OP_BWD)  // delta and -LSE*log2(e), fp32, head-major [h_q, row_pitch] each
-        return align256((size_t)2 * plan->row_pitch * plan->prob.h_q * sizeof(float));
+    // delta and -LSE*log2(e), fp32, head-major [h_q, row_pitch] each
+    const size_t scalars = align256((size_t)2 * plan->row_pitch * plan->prob.h_q * sizeof(float));
+    if (op == BA_OP_BWD) return scalars;
+    if (op == BA_OP_BWD_FUSED)  // plus the fp32 dQ accumulator of the one-kernel backward
+        return scalars + align256((size_t)(plan->prob.n_main + plan->prob.n_branch) * plan->prob.h_q *
+                                  plan->prob.head_dim * sizeof(float));
     return 0;
 }
 
@@ -113,7 +117,8 @@ extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main,
     if (has_main_q && !dQ_main) return BA_EINVAL;
     if (has_branch_q && (!q_branch || !dQ_branch)) return BA_EINVAL;
     if (accumulate != 0 && accumulate != 1) return BA_EINVAL;
-    const size_t need = ba_workspace_bytes(plan, BA_OP_BWD);
+    const bool fused_scratch = (stages & BA_STAGE_FUSED) && !accumulate;
+    const size_t need = ba_workspace_bytes(plan, fused_scratch ? BA_OP_BWD_FUSED : BA_OP_BWD);
     if (!workspace || ws_bytes < need || ((uintptr_t)workspace & 255)) return BA_EWORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     float *delta = (float *)workspace;
@@ -132,8 +137,32 @@ extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main,
     if (!(stages & (BA_STAGE_DQ | BA_STAGE_DKDV | BA_STAGE_FUSED))) return BA_OK;
     const void *qm = has_main_q ? q_main : nullptr;
     if (stages & BA_STAGE_FUSED) {
-        if (plan->impl != BA_IMPL_TC || !accumulate) return BA_EUNSUPPORTED;
-        return ba_tc_bwd_fused(plan, r, qm, q_branch, k, v, delta, dO, accumulate, dQ_main, dQ_branch, dK, dV, st);
+        if (plan->impl != BA_IMPL_TC) return BA_EUNSUPPORTED;
+        if (accumulate)
+            return ba_tc_bwd_fused(plan, r, qm, q_branch, k, v, delta, dO, 1, dQ_main, dQ_branch, dK, dV, st);
+        // gradients in the input dtype: dQ of the selected rows is summed in the workspace, then converted
+        const size_t row_elems = (size_t)hq * d;
+        float *acc_main = (float *)((char *)workspace + ba_workspace_bytes(plan, BA_OP_BWD));
+        float *acc_branch = acc_main + (size_t)n * row_elems;
+        if (has_main_q)
+            BA_CUDA_CHECK(cudaMemsetAsync(acc_main + (size_t)r.qm_begin * row_elems, 0,
+                                          (size_t)(r.qm_end - r.qm_begin) * row_elems * sizeof(float), st));
+        if (has_branch_q)
+            BA_CUDA_CHECK(cudaMemsetAsync(acc_branch + (size_t)r.tok_begin * row_elems, 0,
+                                          (size_t)(r.tok_end - r.tok_begin) * row_elems * sizeof(float), st));
+        rc = ba_tc_bwd_fused(plan, r, qm, q_branch, k, v, delta, dO, 0, acc_main, acc_branch, dK, dV, st);
+        if (rc != BA_OK) return rc;
+        if (has_main_q &&
+            (rc = ba_finalize_grads(acc_main + (size_t)r.qm_begin * row_elems,
+                                    (__nv_bfloat16 *)dQ_main + (size_t)r.qm_begin * row_elems,
+                                    (int64_t)((r.qm_end - r.qm_begin) * row_elems), dt, stream)) != BA_OK)
+            return rc;
+        if (has_branch_q &&
+            (rc = ba_finalize_grads(acc_branch + (size_t)r.tok_begin * row_elems,
+                                    (__nv_bfloat16 *)dQ_branch + (size_t)r.tok_begin * row_elems,
+                                    (int64_t)((r.tok_end - r.tok_begin) * row_elems), dt, stream)) != BA_OK)
+            return rc;
+        return BA_OK;
     }
     if (plan->impl == BA_IMPL_TC)
         return ba_tc_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK,

@@ -77,7 +77,7 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
               const void *k, const void *v, const float *lse, const float *delta,
               const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
               void *dv, cudaStream_t st, int stages);
-// One-kernel backward (ba_tc_bwd_fused.cu): accumulate mode only, dQ by fp32 atomic adds
+// One-kernel backward (ba_tc_bwd_fused.cu): dq_* are fp32 accumulators (atomic adds) in either mode
 int ba_tc_bwd_fused(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
                     const void *k, const void *v, const float *delta, const void *d_o,
                     int accumulate, void *dq_main, void *dq_branch, void *dk, void *dv,

@@ -567,7 +567,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
 int ba_tc_bwd_fused(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
                     const void *v, const float *delta, const void *d_o, int accumulate, void *dq_main,
                     void *dq_branch, void *dk, void *dv, cudaStream_t st) {
-    if (!accumulate) return BA_EUNSUPPORTED;   // dQ is summed into an fp32 accumulator
+    // dq_main / dq_branch are always fp32 accumulators (summed with atomic adds);
+    // `accumulate` says whether dK / dV are fp32 accumulators too or written in bf16
     // the dynamic shared-memory limit is a per-device attribute of the kernel
     static bool attr_set[64] = {};
     int dev = 0;

@@ -51,6 +51,16 @@ def check_fused(ba, oracle, p, seed=0, std=0.5, groups=None, q_main=True, mutate
         if a is not None:
             assert_close(name + " fused vs split", f32(a), f32(b).astype(np.float64), 5e-3)
     plan.check()
+    # gradients in the input dtype: dQ summed in the workspace and converted, dK / dV stored directly
+    gq, gb, gk, gv = ba.branch_attn_bwd(plan, d["q_main"] if q_main else None, d["q_branch"], d["k"], d["v"], o, lse,
+                                        d["d_o"], stages=ba.STAGE_ALL_FUSED)
+    plan.check()
+    assert gb.dtype == torch.bfloat16 and gk.dtype == torch.bfloat16
+    if q_main:
+        assert_close("dQ_main bf16", f32(gq)[:, qh], ref["dq"][:n], tol)
+    assert_close("dQ_branch bf16", f32(gb)[:, qh], ref["dq"][n:], tol)
+    assert_close("dK bf16", f32(gk)[:, kvh], ref["dk"], tol)
+    assert_close("dV bf16", f32(gv)[:, kvh], ref["dv"], tol)
 
 
 @pytest.mark.parametrize("kind", [W.CHAIN, W.BLOCK, W.TREE])
@@ -121,10 +131,15 @@ def test_rejects_what_it_cannot_do(ba):
     d = to_dev(p, W.make_tensors(p, seed=1, std=0.5))
     plan = ba.Plan(p, impl=ba.IMPL_TC)
     o, lse = ba.branch_attn_fwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"])
-    with pytest.raises(ba.BranchAttnError) as e:   # bf16 outputs: no accumulator to add into
-        ba.branch_attn_bwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"], o, lse, d["d_o"],
-                           stages=ba.STAGE_ALL_FUSED)
-    assert e.value.code == -2   # BA_EUNSUPPORTED
+    # gradients in the input dtype need the larger workspace (fp32 dQ accumulator)
+    assert ba._lib().ba_workspace_bytes(plan.handle, ba.OP_BWD_FUSED) > ba._lib().ba_workspace_bytes(plan.handle, ba.OP_BWD)
+    small = plan.workspace(ba.OP_BWD)
+    grads = [torch.empty_like(x) for x in (d["q_main"], d["q_branch"], d["k"], d["v"])]
+    rc = ba._lib().branch_attn_bwd_stages(plan.handle, *(ba._p(x) for x in (d["q_main"], d["q_branch"], d["k"], d["v"], o, lse, d["d_o"])),
+                                          0, p.n_main, 0, p.num_branches, 0, p.n_main, ba.PART_ALL, 0,
+                                          *(ba._p(g) for g in grads), ba._p(small), small.numel(), ba._stream(),
+                                          ba.STAGE_ALL_FUSED)
+    assert rc == -3   # BA_EWORKSPACE
     with pytest.raises(ba.BranchAttnError) as e:   # fused replaces the dQ and dK/dV stages
         ba.branch_attn_bwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"], o, lse, d["d_o"], accumulate=True,
                            stages=ba.STAGE_FUSED | ba.STAGE_DQ)
