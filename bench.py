@@ -238,19 +238,27 @@ def make_device_inputs(p, torch, device, seed=0):
     return t
 
 
-def run_step(rec, plan, t, cp, backward, fused=False):
+def run_fwd(rec, plan, t, cp):
     from paper_2609_07108_b200 import zigzag
     if cp:
         o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp,
                                    out=t.get("_o"), lse=t.get("_lse"))
-        grads = zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp,
-                                fused=fused) if backward else None
-    else:
-        o, lse = rec.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"],
-                                     out=t.get("_o"), lse=t.get("_lse"))
-        grads = rec.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"],
-                                    grads=t.get("_grads"),
-                                    stages=rec.STAGE_ALL_FUSED if fused else rec.STAGE_ALL) if backward else None
+        return o, lse
+    return rec.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], out=t.get("_o"), lse=t.get("_lse"))
+
+
+def run_bwd(rec, plan, t, cp, o, lse, fused=False):
+    from paper_2609_07108_b200 import zigzag
+    if cp:
+        return zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp,
+                               fused=fused)
+    return rec.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"],
+                               grads=t.get("_grads"), stages=rec.STAGE_ALL_FUSED if fused else rec.STAGE_ALL)
+
+
+def run_step(rec, plan, t, cp, backward, fused=False):
+    o, lse = run_fwd(rec, plan, t, cp)
+    grads = run_bwd(rec, plan, t, cp, o, lse, fused=fused) if backward else None
     return o, lse, grads
 
 
@@ -395,7 +403,8 @@ def run_ours(args):
 
 def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     """Same step, inputs in pinned host memory: H2D of Q/K/V/dO, the library
-    calls, D2H of O/LSE and the gradients, all inside the timed region."""
+    calls, D2H of O/LSE and the gradients, all inside the timed region.  The copy
+    of dO overlaps the forward, the copy of O and LSE overlaps the backward."""
     import psutil
     names = tuple(k for k in ("q_main", "q_branch", "k", "v") + (("d_o",) if backward else ()) if t[k] is not None)
     h2d = sum(t[k].numel() * t[k].element_size() for k in names)
@@ -451,14 +460,42 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     s_ev = torch.cuda.Event(enable_timing=True)
     e_ev = torch.cuda.Event(enable_timing=True)
     s_ev.record()
+    # The cotangent is only needed by the backward and O / LSE are final after the
+    # forward: their copies run on side streams behind the forward / the backward.
+    main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    fused = args.bwd == "fused" and plan.impl == ba.IMPL_TC
     for _ in range(steps):
         for k in names:
-            h2d_copy(t[k], k)
-        o, lse, grads = run_step(rec, plan, t, cp, backward, fused=args.bwd == "fused" and plan.impl == ba.IMPL_TC)
-        outs = [o, lse] + (list(grads[:4]) if backward else [])
-        outs = [x for x in outs if x is not None]
-        for i, src in enumerate(outs):
-            d2h_copy(i, src)
+            if k != "d_o":
+                h2d_copy(t[k], k)
+        if backward:
+            qkv_in = torch.cuda.Event()
+            qkv_in.record(main)
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(qkv_in)           # after Q, K, V: the link is theirs first
+                h2d_copy(t["d_o"], "d_o")
+                go_in = torch.cuda.Event()
+                go_in.record(s_in)
+        o, lse = run_fwd(rec, plan, t, cp)
+        outs = [o, lse]
+        if backward:
+            fwd_done = torch.cuda.Event()
+            fwd_done.record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(fwd_done)
+                d2h_copy(0, o)
+                d2h_copy(1, lse)
+                o_out = torch.cuda.Event()
+                o_out.record(s_out)
+            main.wait_event(go_in)
+            grads = run_bwd(rec, plan, t, cp, o, lse, fused=fused)
+            for i, src in enumerate(x for x in grads[:4] if x is not None):
+                d2h_copy(2 + i, src)
+            main.wait_event(o_out)
+        else:
+            d2h_copy(0, o)
+            d2h_copy(1, lse)
     e_ev.record()
     torch.cuda.synchronize()
     ms = s_ev.elapsed_time(e_ev)
