@@ -168,7 +168,7 @@ class Recorder:
         self.events = []           # (kind, start, end)
         self.launches = 0
         self.enabled = False
-        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL", "STAGE_ALL", "STAGE_ALL_FUSED"):
+        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL", "STAGE_ALL", "STAGE_ALL_FUSED", "IMPL_TC"):
             setattr(self, name, getattr(ba, name))
 
     def _wrap(self, kind, n_launch, fn, *a, **k):
@@ -188,6 +188,9 @@ class Recorder:
 
     def branch_attn_fwd_partial(self, *a, **k):
         return self._wrap("fwd", 1, self.ba.branch_attn_fwd_partial, *a, **k)
+
+    def branch_attn_fwd_partial_merge(self, *a, **k):
+        return self._wrap("fwd", 1, self.ba.branch_attn_fwd_partial_merge, *a, **k)
 
     def lse_merge(self, *a, **k):
         return self._wrap("lse_merge", 1, self.ba.lse_merge, *a, **k)
@@ -376,7 +379,9 @@ def run_ours(args):
             "dtype": p.dtype, "data": "synthetic",
             "config": {"workload": name, "n_main": p.n_main, "rows": p.rows, "h_q": p.h_q, "h_kv": p.h_kv,
                        "head_dim": p.head_dim, "mask": W.KIND_NAMES[p.kind], "pairs_per_head": pairs,
-                       "path": (f"zigzag cp={cp}: partial fwd + lse_merge, partial bwd accumulate"
+                       "path": (f"zigzag cp={cp}: partial fwd merged by Eq. lse-merge "
+                                + ("in the kernel epilogue" if plan.impl == ba.IMPL_TC else "with lse_merge")
+                                + ", partial bwd accumulate"
                                 if cp else "monolithic fwd + bwd"),
                        "backward": backward,
                        "bwd_kernels": ("one fused kernel (dQ by fp32 atomic adds)" if fused

@@ -151,6 +151,20 @@ int branch_attn_fwd_partial(const ba_plan_t *plan, const void *q_main, const voi
                             void *workspace, size_t ws_bytes, void *stream);
 
 /*
+ * The same partial forward with Eq. (lse-merge) applied in the kernel's epilogue:
+ * (O_acc, LSE_acc), compact fp32 as above and holding the result of the key sets
+ * seen so far (first filled by branch_attn_fwd_partial), are replaced by their
+ * merge with this call's partial result.  Saves the separate lse_merge pass of a
+ * ring step.  Tensor-core plans only (BA_EUNSUPPORTED otherwise).
+ */
+int branch_attn_fwd_partial_merge(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                                  const void *k, const void *v,
+                                  int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                                  int64_t kv_begin, int64_t kv_end, int parts,
+                                  float *O_acc, float *LSE_acc,
+                                  void *workspace, size_t ws_bytes, void *stream);
+
+/*
  * Eq. (lse-merge):  l = log(e^la + e^lb),  O = e^(la-l) Oa + e^(lb-l) Ob,
  * evaluated in max-subtracted form; la = lb = -inf gives l = -inf, O = 0.
  *   rows_heads = number of (row, head) pairs; O_a/O_b fp32 [rows_heads, d],

@@ -47,7 +47,7 @@ class _Problem(C.Structure):
 _LIB = None
 EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
            "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "ba_plan_check", "branch_attn_fwd",
-           "branch_attn_fwd_partial", "lse_merge", "branch_attn_bwd", "branch_attn_bwd_stages",
+           "branch_attn_fwd_partial", "branch_attn_fwd_partial_merge", "lse_merge", "branch_attn_bwd", "branch_attn_bwd_stages",
            "branch_attn_bwd_static", "ba_finalize_grads")
 
 
@@ -84,6 +84,8 @@ def _lib():
         lib.branch_attn_fwd_partial.restype = C.c_int
         lib.branch_attn_fwd_partial.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64,
                                                 C.c_int, vp, vp, vp, C.c_size_t, vp]
+        lib.branch_attn_fwd_partial_merge.restype = C.c_int
+        lib.branch_attn_fwd_partial_merge.argtypes = lib.branch_attn_fwd_partial.argtypes
         lib.lse_merge.restype = C.c_int
         lib.lse_merge.argtypes = [i64, C.c_int, vp, vp, vp, vp, vp, C.c_int, vp, vp]
         lib.branch_attn_bwd.restype = C.c_int
@@ -220,6 +222,17 @@ def branch_attn_fwd_partial(plan, q_main, q_branch, k, v, qm_range, br_range, kv
                                         _p(ws), ws.numel(), _stream())
     _check(rc, "branch_attn_fwd_partial")
     return out, lse
+
+
+def branch_attn_fwd_partial_merge(plan, q_main, q_branch, k, v, qm_range, br_range, kv_range, parts, acc_o, acc_lse):
+    """Partial forward whose epilogue merges into the compact fp32 (acc_o, acc_lse) in place."""
+    ws = plan.workspace(OP_FWD)
+    rc = _lib().branch_attn_fwd_partial_merge(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v),
+                                              qm_range[0], qm_range[1], br_range[0], br_range[1],
+                                              kv_range[0], kv_range[1], parts, _p(acc_o), _p(acc_lse),
+                                              _p(ws), ws.numel(), _stream())
+    _check(rc, "branch_attn_fwd_partial_merge")
+    return acc_o, acc_lse
 
 
 def lse_merge(o_a, lse_a, o_b, lse_b, out=None, lse_out=None, out_dtype=torch.float32):

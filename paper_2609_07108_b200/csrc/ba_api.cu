@@ -49,7 +49,7 @@ extern "C" size_t ba_workspace_bytes(const ba_plan_t *plan, int op) {
 }
 
 static int fwd_common(const ba_plan_t *plan, const BaRange &r, const void *q_main, const void *q_branch,
-                      const void *k, const void *v, void *o, float *lse, bool partial, void *stream) {
+                      const void *k, const void *v, void *o, float *lse, int partial, void *stream) {
     const bool has_main_q = q_main != nullptr && r.qm_end > r.qm_begin;
     const bool has_branch_q = r.tok_end > r.tok_begin;
     if (!has_main_q && !has_branch_q) return BA_OK;
@@ -57,7 +57,8 @@ static int fwd_common(const ba_plan_t *plan, const BaRange &r, const void *q_mai
     if (has_branch_q && !q_branch) return BA_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     if (plan->impl == BA_IMPL_TC) return ba_tc_fwd(plan, r, q_main, q_branch, k, v, o, lse, partial, st);
-    return ba_simt_fwd(plan, r, q_main, q_branch, k, v, o, lse, partial, st);
+    if (partial == 2) return BA_EUNSUPPORTED;   // merge in the epilogue: tensor-core kernel only
+    return ba_simt_fwd(plan, r, q_main, q_branch, k, v, o, lse, partial != 0, st);
 }
 
 extern "C" int branch_attn_fwd(const ba_plan_t *plan, const void *q_main, const void *q_branch,
@@ -69,7 +70,7 @@ extern "C" int branch_attn_fwd(const ba_plan_t *plan, const void *q_main, const 
     int rc = make_range(plan, 0, plan->prob.n_main, 0, plan->prob.num_branches, 0, plan->prob.n_main,
                         BA_PART_MAIN | BA_PART_BRANCH, &r);
     if (rc != BA_OK) return rc;
-    return fwd_common(plan, r, q_main, q_branch, k, v, O, LSE, false, stream);
+    return fwd_common(plan, r, q_main, q_branch, k, v, O, LSE, 0, stream);
 }
 
 extern "C" int branch_attn_fwd_partial(const ba_plan_t *plan, const void *q_main, const void *q_branch,
@@ -83,7 +84,21 @@ extern "C" int branch_attn_fwd_partial(const ba_plan_t *plan, const void *q_main
     int rc = make_range(plan, qm_begin, qm_end, br_begin, br_end, kv_begin, kv_end, parts, &r);
     if (rc != BA_OK) return rc;
     if (!q_main && qm_end > qm_begin) return BA_EINVAL;
-    return fwd_common(plan, r, q_main, q_branch, k, v, O_part, LSE_part, true, stream);
+    return fwd_common(plan, r, q_main, q_branch, k, v, O_part, LSE_part, 1, stream);
+}
+
+extern "C" int branch_attn_fwd_partial_merge(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                                             const void *k, const void *v, int64_t qm_begin, int64_t qm_end,
+                                             int64_t br_begin, int64_t br_end, int64_t kv_begin,
+                                             int64_t kv_end, int parts, float *O_acc, float *LSE_acc,
+                                             void *workspace, size_t ws_bytes, void *stream) {
+    (void)workspace; (void)ws_bytes;
+    if (!plan) return BA_EINVAL;
+    BaRange r;
+    int rc = make_range(plan, qm_begin, qm_end, br_begin, br_end, kv_begin, kv_end, parts, &r);
+    if (rc != BA_OK) return rc;
+    if (!q_main && qm_end > qm_begin) return BA_EINVAL;
+    return fwd_common(plan, r, q_main, q_branch, k, v, O_acc, LSE_acc, 2, stream);
 }
 
 extern "C" int branch_attn_bwd(const ba_plan_t *plan, const void *q_main, const void *q_branch,

@@ -70,8 +70,9 @@ int ba_simt_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const v
                 const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
                 void *dv, cudaStream_t st, int stages);
 // Tensor-core path (ba_tc_fwd.cu / ba_tc_bwd.cu)
+// partial_out: 0 = final layout in the input dtype, 1 = compact fp32, 2 = compact fp32 merged in place
 int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
-              const void *k, const void *v, void *o, float *lse, bool partial_out,
+              const void *k, const void *v, void *o, float *lse, int partial_out,
               cudaStream_t st);
 int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
               const void *k, const void *v, const float *lse, const float *delta,

@@ -66,6 +66,23 @@ __device__ __forceinline__ uint64_t bit_range(int lo, int hi) {
     return (~0ull >> (63 - hi)) & (~0ull << lo);
 }
 
+// Eq. (lse-merge) on one 32-column chunk of an fp32 row: dst = dst * w_old + r * w_new
+// (dst is not read when w_old is 0: it may be uninitialised then)
+__device__ __forceinline__ void merge_row_chunk(void *o, size_t elem_off, const uint32_t (&r)[32], float w_new,
+                                                float w_old) {
+    float4 *dst = reinterpret_cast<float4 *>((float *)o + elem_off);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (w_old != 0.f) a = dst[i];
+        a.x = a.x * w_old + __uint_as_float(r[4 * i]) * w_new;
+        a.y = a.y * w_old + __uint_as_float(r[4 * i + 1]) * w_new;
+        a.z = a.z * w_old + __uint_as_float(r[4 * i + 2]) * w_new;
+        a.w = a.w * w_old + __uint_as_float(r[4 * i + 3]) * w_new;
+        dst[i] = a;
+    }
+}
+
 template <bool OUT_F32>
 __device__ __forceinline__ void store_row_chunk(void *o, size_t elem_off, const uint32_t (&r)[32], float inv) {
     if (OUT_F32) {
@@ -439,8 +456,24 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 orow = is_main ? my_row - p.r.qm_begin : (p.r.qm_end - p.r.qm_begin) + (my_row - p.r.tok_begin);
             const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
             const size_t base = ((size_t)orow * p.h_q + h) * 128;
-            if (do_store)
-                p.lse[orow * p.h_q + h] = l_run > 0.f ? (m_run * sl2 + log2f(l_run)) * kLn2 : -INFINITY;
+            const float lse_p = l_run > 0.f ? (m_run * sl2 + log2f(l_run)) * kLn2 : -INFINITY;
+            float w_new = inv, w_old = 0.f;   // partial_out == 2: weights of Eq. (lse-merge)
+            if (do_store) {
+                float lse_out = lse_p;
+                if (p.partial_out == 2) {
+                    const float lse_a = p.lse[orow * p.h_q + h];
+                    const float mx = fmaxf(lse_a, lse_p);
+                    if (mx == -INFINITY) {
+                        lse_out = -INFINITY; w_new = 0.f;
+                    } else {
+                        const float ea = expf(lse_a - mx), ep = expf(lse_p - mx), s = ea + ep;
+                        lse_out = mx + logf(s);
+                        w_old = ea / s;
+                        w_new = ep / s * inv;
+                    }
+                }
+                p.lse[orow * p.h_q + h] = lse_out;
+            }
             // every lane runs the (warp-collective) TMEM loads; only live rows store
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -453,7 +486,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                     for (int e = 0; e < 32; ++e) r[e] = 0u;
                 }
                 if (do_store) {
-                    if (p.partial_out) store_row_chunk<true>(p.o, base + c * 32, r, inv);
+                    if (p.partial_out == 2) merge_row_chunk(p.o, base + c * 32, r, w_new, w_old);
+                    else if (p.partial_out) store_row_chunk<true>(p.o, base + c * 32, r, inv);
                     else store_row_chunk<false>(p.o, base + c * 32, r, inv);
                 }
             }
@@ -473,7 +507,7 @@ bool ba_tc_supported(const ba_problem_t *p) {
 }
 
 int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
-              const void *v, void *o, float *lse, bool partial_out, cudaStream_t st) {
+              const void *v, void *o, float *lse, int partial_out, cudaStream_t st) {
     // the dynamic shared-memory limit is a per-device attribute of the kernel
     static bool attr_set[64] = {};
     int dev = 0;
@@ -496,7 +530,7 @@ int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
     p.group = pr.h_q / pr.h_kv;
     p.pairs_per_group = (p.group + 1) / 2;
     p.scale_log2 = pl->scale * kLog2e;
-    p.partial_out = partial_out ? 1 : 0;
+    p.partial_out = partial_out;   // 0 final layout, 1 compact fp32, 2 compact fp32 merged in place
     p.status = pl->dev_status;
     const int64_t mt = q_main ? (r.qm_end - r.qm_begin + kTile - 1) / kTile : 0;
     const int64_t bt = (r.tok_end - r.tok_begin + kTile - 1) / kTile;

@@ -93,7 +93,9 @@ def pairs_per_rank(problem, cp: int) -> List[int]:
 
 
 def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None):
-    """Emulated CP forward: per (rank, step) partial calls + lse_merge.
+    """Emulated CP forward: per (rank, step) partial calls, each merged into the
+    running (O, LSE) by Eq. (lse-merge) -- in the kernel's epilogue on tensor-core
+    plans, by `lse_merge` otherwise.
     Returns (O [N+M,h_q,D] input dtype, LSE fp32, number of library launches)."""
     import torch
     p = plan.problem
@@ -112,16 +114,24 @@ def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None):
         max_rows = max(max_rows, csize + t1 - t0)
     acc_o = torch.empty((max_rows, p.h_q, p.head_dim), dtype=torch.float32, device=plan.device)
     acc_l = torch.empty((max_rows, p.h_q), dtype=torch.float32, device=plan.device)
-    inc_o = torch.empty_like(acc_o)
-    inc_l = torch.empty_like(acc_l)
+    # tensor-core plans merge each later ring step into the accumulators in the kernel's
+    # epilogue; the plain-FMA path writes the step's partial result and merges it in a pass of its own
+    in_kernel = plan.impl == ba.IMPL_TC
+    inc_o = None if in_kernel else torch.empty_like(acc_o)
+    inc_l = None if in_kernel else torch.empty_like(acc_l)
     for rank in range(cp):
         for qc in rank_chunks(rank, cp):
             mine = [b for b in blocks if b.rank == rank and b.q_chunk == qc]
             t0, t1 = plan.token_range(*mine[0].br)
             rows = csize + t1 - t0
-            a_o, a_l, i_o, i_l = acc_o[:rows], acc_l[:rows], inc_o[:rows], inc_l[:rows]
+            a_o, a_l = acc_o[:rows], acc_l[:rows]
             for j, b in enumerate(mine):
                 parts = ba.PART_MAIN | (ba.PART_BRANCH if b.branch_part else 0)
+                if j > 0 and in_kernel:
+                    ba.branch_attn_fwd_partial_merge(plan, q_main, q_branch, k, v, b.qm, b.br, b.kv, parts, a_o, a_l)
+                    launches += 1
+                    continue
+                i_o, i_l = (None, None) if in_kernel else (inc_o[:rows], inc_l[:rows])
                 dst = (a_o, a_l) if j == 0 else (i_o, i_l)
                 ba.branch_attn_fwd_partial(plan, q_main, q_branch, k, v, b.qm, b.br, b.kv, parts,
                                            out=dst[0], lse=dst[1])

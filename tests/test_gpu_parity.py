@@ -254,3 +254,46 @@ def test_partial_chunks_merge_to_monolithic(ba, oracle, dtype, d):
             assert_close(name + " finalized", f32(fin), w, tol)
             assert_close(name + " monolithic", f32(g_mono), w, tol)
     torch.cuda.synchronize()
+
+
+def test_partial_forward_merged_in_the_epilogue(ba, oracle):
+    """Ring steps whose (O, LSE) are merged into the running result inside the kernel
+    (Eq. lse-merge in the epilogue) against the oracle's monolithic forward, on chunks
+    that leave rows without any visible key, then give them some."""
+    p = W.odd_shapes(W.TREE, head_dim=128, dtype="bf16")
+    t = W.make_tensors(p, seed=13, std=0.5)
+    d = to_dev(p, t)
+    n, a = p.n_main, p.num_branches
+    plan = ba.Plan(p, impl=ba.IMPL_TC)
+    ref = oracle_fwd_bwd(oracle, p, t, backward=False)
+    for qm, br in (((0, n), (0, a)), ((37, 300), (2, a - 1))):
+        t0, t1 = plan.token_range(*br)
+        rows = np.concatenate([np.arange(qm[0], qm[1]), n + np.arange(t0, t1)])
+        acc = None
+        # the branch part first or last, an empty chunk, one-key chunks
+        for order in (0, 1):
+            chunks = [(150, n), (0, 17), (17, 18), (150, 150), (18, 150)]
+            acc = None
+            for i, kv in enumerate(chunks):
+                parts = ba.PART_MAIN | (ba.PART_BRANCH if i == (0 if order == 0 else 4) else 0)
+                if acc is None:
+                    acc = ba.branch_attn_fwd_partial(plan, d["q_main"], d["q_branch"], d["k"], d["v"], qm, br, kv, parts)
+                else:
+                    ba.branch_attn_fwd_partial_merge(plan, d["q_main"], d["q_branch"], d["k"], d["v"], qm, br, kv,
+                                                     parts, acc[0], acc[1])
+            plan.check()
+            assert_close(f"merged O (order {order})", f32(acc[0]), ref["o"][rows], TOL["bf16"])
+            assert_lse_close(f32(acc[1]), ref["lse"][rows])
+    # a key set that no selected row sees at all: -inf and zeros, and merging into it works
+    acc = ba.branch_attn_fwd_partial(plan, d["q_main"], d["q_branch"], d["k"], d["v"], (0, 10), (0, 0), (200, n), ba.PART_MAIN)
+    assert torch.isneginf(acc[1]).all() and float(acc[0].abs().max()) == 0.0
+    ba.branch_attn_fwd_partial_merge(plan, d["q_main"], d["q_branch"], d["k"], d["v"], (0, 10), (0, 0), (0, 200),
+                                     ba.PART_MAIN, acc[0], acc[1])
+    plan.check()
+    assert_close("merge into an empty result", f32(acc[0]), ref["o"][:10], TOL["bf16"])
+    assert_lse_close(f32(acc[1]), ref["lse"][:10])
+    simt = ba.Plan(p, impl=ba.IMPL_SIMT)
+    with pytest.raises(ba.BranchAttnError) as e:
+        ba.branch_attn_fwd_partial_merge(simt, d["q_main"], d["q_branch"], d["k"], d["v"], (0, 10), (0, 0), (0, 200),
+                                         ba.PART_MAIN, acc[0], acc[1])
+    assert e.value.code == -2   # BA_EUNSUPPORTED
