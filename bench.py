@@ -42,6 +42,8 @@ WORKLOADS = {
     "config4_tree_64k": (4, 1, 0, True),
     "config3_dflash_32k": (3, 1, 0, True),
     "config2_eagle3_8k": (2, 1, 0, False),
+    # shape of the paper's packed variable-length operator benchmark (longest sequence 20,480 tokens)
+    "varlen_ttt_72k": (6, 1, 0, True),
 }
 
 

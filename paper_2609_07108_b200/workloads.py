@@ -219,7 +219,23 @@ def config5(shrink: int = 1) -> Problem:
                    32, 8, 128, name=f"config5_long_chain_{total}", extra={"cp": 8})
 
 
-CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
+def varlen_ttt(shrink: int = 1) -> Problem:
+    """Shape of the paper's operator benchmark (Section 4.4): a packed
+    variable-length batch whose longest sequence has 20,480 tokens and whose
+    padded-to-longest size is about 2.25 times its real size, EAGLE-3
+    training-time test with three draft passes (depth-3 chain at every
+    position).  Eight sequences, 73,728 tokens; the paper gives no length
+    distribution beyond those two figures."""
+    lens = [20480, 14336, 11264, 9216, 7168, 5120, 4096, 2048]
+    lens = [max(1, x // shrink) for x in lens]
+    total = int(sum(lens))
+    cu = cu_from_lengths(lens)
+    anchors = np.arange(total, dtype=np.int32)
+    return Problem(cu, anchors, uniform_branch_offsets(total, 3), CHAIN, None,
+                   32, 8, 128, name=f"varlen_ttt_chain_{total}")
+
+
+CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5, 6: varlen_ttt}
 
 
 def odd_shapes(kind: int, seed: int = 0, h_q: int = 4, h_kv: int = 2, head_dim: int = 64,

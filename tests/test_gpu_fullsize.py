@@ -158,6 +158,13 @@ def test_config4_full_size(ba, oracle):
     check_sampled(ba, oracle, p, cp=0, groups=[2, 5], n_rows=512, seed=2, edges=tile_edges(p))
 
 
+def test_varlen_ttt_full_size(ba, oracle):
+    """The paper's packed variable-length operator-benchmark shape (eight sequences, longest 20,480 tokens)."""
+    p = W.varlen_ttt()
+    assert p.n_main == 73728 and int(np.diff(p.cu_seqlens).max()) == 20480
+    check_sampled(ba, oracle, p, cp=0, groups=[0, 7], n_rows=256, seed=5, edges=tile_edges(p))
+
+
 @pytest.mark.parametrize("fused", [False, True], ids=["split_bwd", "fused_bwd"])
 def test_config5_full_size_zigzag(ba, oracle, fused):
     """256K tokens through the emulated 8-way zigzag layout: partial forward +

@@ -68,7 +68,7 @@ def test_odd_shapes_all_masks(ba, oracle, kind):
     check_fused(ba, oracle, W.odd_shapes(kind, head_dim=128, dtype="bf16"), seed=3)
 
 
-@pytest.mark.parametrize("cfg,shrink", [(3, 16), (4, 16), (5, 128)])
+@pytest.mark.parametrize("cfg,shrink", [(3, 16), (4, 16), (5, 128), (6, 64)])
 def test_shrunken_configs(ba, oracle, cfg, shrink):
     p = W.CONFIGS[cfg](shrink)
     check_fused(ba, oracle, p, seed=0, groups=[0, p.h_kv - 1])

@@ -137,7 +137,7 @@ def test_branch_queries_only(ba, oracle, kind):
         check_full(ba, oracle, p, seed=4, std=0.5, impl=impl, q_main=False)
 
 
-@pytest.mark.parametrize("cfg,shrink", [(2, 8), (3, 16), (4, 16), (5, 128)])
+@pytest.mark.parametrize("cfg,shrink", [(2, 8), (3, 16), (4, 16), (5, 128), (6, 64)])
 def test_shrunken_configs_bf16(ba, oracle, cfg, shrink):
     p = W.CONFIGS[cfg](shrink)
     for impl in impls_for(ba, p):
