@@ -49,12 +49,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ uint64_t global_timer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
 // Bounded wait: gives up after `kWaitLimitNs` (a legitimate wait in these
 // kernels lasts microseconds) or as soon as another thread of the CTA raised
 // `*abort_flag`; then raises the flag itself and returns false, so that every
@@ -143,25 +137,6 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar) {
                  : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
 // 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives
 // columns [col, col + 32) of TMEM lane (lane base of the warp) + i.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -215,25 +190,16 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 
 // --------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor for 128-byte-swizzled tiles (as TMA writes
-// them with CU_TENSOR_MAP_SWIZZLE_128B into 1024-byte aligned buffers).
+// them with CU_TENSOR_MAP_SWIZZLE_128B into 1024-byte aligned buffers), kept as
+// its two 32-bit words.  Bits: address >> 4 in [0,14), leading byte offset >> 4 in
+// [16,30), stride byte offset >> 4 in [32,46), descriptor version 1 at bit 46,
+// swizzle mode 2 (128 bytes) in [61,64).
 //   K-major operand  (rows = M or N index, 64 bf16 of K per 128-byte row):
-//     sbo = 1024 (next group of 8 rows), lbo unused.
+//     sbo = 1024 (next group of 8 rows), lbo unused (16).
 //   MN-major operand (rows = K index, 64 bf16 of M/N per 128-byte row):
 //     sbo = 1024 (next group of 8 K rows), lbo = distance to the next block of
 //     64 M/N elements.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes,
-                                                    uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;  // 128-byte swizzle
-    return d;
-}
-
-// The same descriptor as two 32-bit words.  Only the low word holds the address
-// (bits 0-13, in 16-byte units), so the issuing thread keeps one low word per
+// Only the low word holds the address, so the issuing thread keeps one low word per
 // operand and advances it with a 32-bit add per MMA instead of rebuilding the
 // descriptor: one thread issues every MMA of a CTA, and with rebuilt descriptors
 // that thread, not the tensor core, set the pace (about 81 instead of 64 clocks

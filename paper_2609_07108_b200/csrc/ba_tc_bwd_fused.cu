@@ -221,7 +221,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
     const int n_sub_main = m1 > m0 ? (int)((m1 - ma + kTile - 1) / kTile) : 0;
     const int n_sub_br = b1 > b0 ? (int)((b1 - ba + kTile - 1) / kTile) : 0;
     const int n_sub = n_sub_main + n_sub_br;
-    const int n_iter = n_sub * p.group;   // t = head_in_group * n_sub + s
+    // t = head_in_group * n_sub + s, and step s works on tile n_sub - 1 - s: every key tile's query
+    // range ends where its sequence (or the call's query range) ends, so CTAs that start together
+    // walk the same tiles at the same time from that common end and share them through L2,
+    // whereas their first tiles differ (causal: key tile k starts at row tile k)
+    const int n_iter = n_sub * p.group;
 
     if (warp >= 12) {
       reg_dec<kRegsIssue>();
@@ -247,8 +251,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                 if (t >= 2) ok = mbar_wait(&sm.q_empty[st], ((t >> 1) - 1) & 1, abort_flag);
                 if (!ok) break;
                 const int h = g * p.group + hh;
-                const bool seg_main = s < n_sub_main;
-                const int64_t r0 = seg_main ? ma + (int64_t)s * kTile : ba + (int64_t)(s - n_sub_main) * kTile;
+                const int u = n_sub - 1 - s;   // tiles are walked from the last one down (see n_iter)
+                const bool seg_main = u < n_sub_main;
+                const int64_t r0 = seg_main ? ma + (int64_t)u * kTile : ba + (int64_t)(u - n_sub_main) * kTile;
                 const int64_t grow0 = seg_main ? r0 : n + r0;
                 const CUtensorMap *tq = seg_main ? &tm_q_main : &tm_q_branch;
                 mbar_expect_tx(&sm.q_full[st], 2 * kTileBytes + 2 * kTile * 4);
@@ -262,8 +267,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                 issued = t + 1;
                 if (t + kPrefetch < n_iter) {
                     const int h2 = g * p.group + ph;
-                    const bool main2 = ps < n_sub_main;
-                    const int64_t r2 = main2 ? ma + (int64_t)ps * kTile : ba + (int64_t)(ps - n_sub_main) * kTile;
+                    const int u2 = n_sub - 1 - ps;
+                    const bool main2 = u2 < n_sub_main;
+                    const int64_t r2 = main2 ? ma + (int64_t)u2 * kTile : ba + (int64_t)(u2 - n_sub_main) * kTile;
                     const int64_t g2 = main2 ? r2 : n + r2;
                     const CUtensorMap *tq2 = main2 ? &tm_q_main : &tm_q_branch;
                     for (int half = 0; half < 2; ++half) {
@@ -398,8 +404,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
         const float sc = p.scale;
         int s = 0, hh = 0;                              // tile t = hh * n_sub + s
         for (int t = 0; t < n_iter; ++t) {
-            const bool seg_main = s < n_sub_main;
-            const int r0 = seg_main ? (int)ma + s * kTile : (int)ba + (s - n_sub_main) * kTile;   // first query row
+            const int u = n_sub - 1 - s;
+            const bool seg_main = u < n_sub_main;
+            const int r0 = seg_main ? (int)ma + u * kTile : (int)ba + (u - n_sub_main) * kTile;   // first query row
             const int rbeg = seg_main ? (int)m0 : (int)b0, rend = seg_main ? (int)m1 : (int)b1;
             const int c_lo = max(rbeg - r0, 0), c_hi = min(rend - r0, kTile);
             float *ptr = (float *)(seg_main ? p.dq_main : p.dq_branch) +
@@ -454,8 +461,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
         const int ma_i = (int)ma + 64 * hf, ba_i = (int)ba + 64 * hf;
         for (int t = 0; t < n_iter; ++t) {
             const int st = t & 1;
-            const bool seg_main = s < n_sub_main;
-            const int r0h = seg_main ? ma_i + s * kTile : ba_i + (s - n_sub_main) * kTile;   // my first query row
+            const int u = n_sub - 1 - s;
+            const bool seg_main = u < n_sub_main;
+            const int r0h = seg_main ? ma_i + u * kTile : ba_i + (u - n_sub_main) * kTile;   // my first query row
             const int rbeg = seg_main ? (int)m0 : (int)b0, rend = seg_main ? (int)m1 : (int)b1;
             // --- which of my 64 query rows (columns) see my key
             uint64_t vis = 0ull;
