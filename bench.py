@@ -47,6 +47,15 @@ WORKLOADS = {
 }
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the launches of
+# one step) from a one-pass ncu capture of the full-size command; not measurable live.  The command
+# and the per-launch breakdown are in profiles/dram_traffic_config5_256k_zigzag.md.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("config5_256k_zigzag", "tc_bwd_fused_kernel"): 11.36e9,
+    ("config5_256k_zigzag_fwd", "tc_fwd_kernel"): 5.68e9,
+}
+
+
 def useful_flops(p, backward=True, branch_only=False):
     pairs = W.useful_pairs(p, with_main_queries=not branch_only)
     per_pair = 4 * p.head_dim * p.h_q
@@ -359,7 +368,8 @@ def run_ours(args):
             peak = peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"]
             roof = {"bound": "tensor", "kernel": kernel_name, "flop_per_pair_head": share * p.head_dim,
                     "achieved": round(achieved, 2), "peak": peak,
-                    "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": None,
+                    "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
+                    "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((name, kernel_name)),
                     "peak_source": f"{peaks['_source']} {'sustained' if long_step else 'burst'} bf16",
                     "launches": calls, "avg_launch_ms": round(ms / calls, 4),
                     "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
