@@ -84,6 +84,56 @@ def test_branch_queries_only(ba, oracle, kind):
     check_fused(ba, oracle, W.odd_shapes(kind, head_dim=128, dtype="bf16"), seed=4, q_main=False)
 
 
+def _sharp(t):          # near one-hot softmax rows
+    t["q_main"] *= 8
+    t["q_branch"] *= 8
+
+
+def _offset(t):         # a large common component in every key: scores far from zero
+    rng = np.random.default_rng(99)
+    c = W.round_to_bf16(rng.standard_normal(t["k"].shape[-1]).astype(np.float32) * 4)
+    t["k"] += c
+    t["k"][:] = W.round_to_bf16(t["k"])
+
+
+def _late_outlier(t):   # one key aligned with a late query
+    t["k"][400] = W.round_to_bf16(t["q_main"][404, 0] * 3)
+
+
+@pytest.mark.parametrize("mutate", [_sharp, _offset, _late_outlier])
+def test_stress_inputs(ba, oracle, mutate):
+    p = W.odd_shapes(W.CHAIN, head_dim=128, dtype="bf16", h_q=4, h_kv=2)
+    check_fused(ba, oracle, p, seed=6, mutate=mutate)
+
+
+def test_unaligned_ranges_with_gradients_in_the_input_dtype(ba, oracle):
+    """Query and key ranges that start and end inside tiles; rows and keys outside the
+    ranges keep what the output tensors held."""
+    p = W.odd_shapes(W.BLOCK, head_dim=128, dtype="bf16")
+    t = W.make_tensors(p, seed=15, std=0.5)
+    d = to_dev(p, t)
+    n, a = p.n_main, p.num_branches
+    plan = ba.Plan(p, impl=ba.IMPL_TC)
+    o, lse = ba.branch_attn_fwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"])
+    qm, br, kv = (37, 301), (1, a - 1), (13, 333)
+    t0, t1 = plan.token_range(*br)
+    rows = np.concatenate([np.arange(*qm), n + np.arange(t0, t1)])
+    ref_dq, ref_dk, ref_dv = oracle.backward(p, oracle.gather_q(p, t["q_main"], t["q_branch"], rows), t["k"], t["v"],
+                                             t["d_o"][rows], rows=rows, parts=3, kv_range=kv)
+    grads = tuple(torch.full(x.shape, 7.0, dtype=torch.bfloat16, device="cuda")
+                  for x in (d["q_main"], d["q_branch"], d["k"], d["v"]))
+    ba.branch_attn_bwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"], o, lse, d["d_o"], qm_range=qm, br_range=br,
+                       kv_range=kv, grads=grads, stages=ba.STAGE_ALL_FUSED)
+    plan.check()
+    dq = torch.cat([grads[0], grads[1]], 0)
+    assert_close("dQ (selected rows)", f32(dq)[rows], ref_dq, TOL["bf16"])
+    other = np.ones(p.rows, bool); other[rows] = False
+    assert float((dq[torch.from_numpy(other).cuda()].float() - 7.0).abs().max()) == 0.0
+    keys = np.concatenate([np.arange(*kv), n + np.arange(t0, t1)])       # the key set of the call
+    assert_close("dK (key set)", f32(grads[2])[keys], ref_dk[keys], TOL["bf16"])
+    assert_close("dV (key set)", f32(grads[3])[keys], ref_dv[keys], TOL["bf16"])
+
+
 def test_no_branches(ba, oracle):
     cu = W.cu_from_lengths([100, 300, 29])
     p = W.Problem(cu, np.zeros(0, np.int32), np.zeros(1, np.int32), W.CHAIN, None, 4, 2, 128, dtype="bf16")
