@@ -4,9 +4,10 @@
 // accumulated over key chunks), but S and dP are formed once per (key tile,
 // query tile, head) instead of once in a dQ kernel and once in a dK/dV kernel:
 // 10 D flop per visible pair instead of 14 D.  The price: dQ rows are shared by
-// all key tiles, so they are summed with fp32 atomic adds into an accumulator
-// (`accumulate` mode only) and their rounding depends on the arrival order;
-// dK and dV still have one owning CTA and stay bit-reproducible.
+// all key tiles, so they are summed with fp32 atomic adds into an accumulator (the
+// caller's in `accumulate` mode, one in the workspace otherwise) and their
+// rounding depends on the arrival order; dK and dV still have one owning CTA and
+// stay bit-reproducible.
 //
 // Key-stationary: one CTA owns 128 key rows of one KV head, keeps K_j, V_j in
 // shared memory and dK_j, dV_j (fp32) in TMEM, and walks the query rows that can
