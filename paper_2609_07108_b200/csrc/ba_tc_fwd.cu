@@ -40,7 +40,7 @@ struct FwdSmem {
     alignas(1024) uint8_t kv[kStages][kTileBytes];
     alignas(8) uint64_t q_full;
     uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2], p_half[2], p_full[2], o_full[2];
     uint32_t tmem_base;
     int abort_flag;
     int lo_min, hi_max, lo_max, hi_min, bs_min, be_max;
@@ -173,6 +173,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
         for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.s_full[i], 1);
+            mbar_init(&sm.p_half[i], 128);
             mbar_init(&sm.p_full[i], 128);
             mbar_init(&sm.o_full[i], 1);
         }
@@ -288,10 +289,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 for (int ks = 0; ks < 8; ++ks)
                     mma_ss_lh(tmem + i * 128, q_km[i] + desc_step_kmajor(ks), k_km + desc_step_kmajor(ks), IDESC_QK, ks > 0);
             };
-            auto issue_pv = [&](int i, int stage, bool accumulate) {
+            auto issue_pv = [&](int i, int stage, bool accumulate, int ks0) {   // K steps ks0 .. ks0 + 3
                 const uint32_t v_mn = kv_mn0 + stage * kStageStep;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
+                for (int ks = ks0; ks < ks0 + 4; ++ks)
                     mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, v_mn + desc_step_mnmajor(ks), IDESC_PV,
                               accumulate || ks > 0);
             };
@@ -307,11 +308,15 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 const int it_v = 2 * j + 1, sv = it_v % kStages;
                 const int it_k = 2 * j + 2, sk = it_k % kStages;
                 for (int i = 0; i < 2 && ok; ++i) {
-                    ok = mbar_wait(&sm.p_full[i], j & 1, abort_flag);
+                    ok = mbar_wait(&sm.p_half[i], j & 1, abort_flag);
                     if (ok && i == 0) ok = mbar_wait(&sm.kv_full[sv], (it_v / kStages) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(i, sv, j > 0);
+                    issue_pv(i, sv, j > 0, 0);            // keys 0-63 while the softmax warps finish keys 64-127
+                    ok = mbar_wait(&sm.p_full[i], j & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(i, sv, true, 4);
                     if (i == 1) tc_commit(&sm.kv_empty[sv]);
                     if (j + 1 < T) {
                         if (i == 0) {
@@ -421,6 +426,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 chunk_exp<true>(rb, mk1, sl2, neg_ms, l2, pk);
                 tmem_st16(s_addr + 16, pk);
                 tmem_ld32(s_addr + 96, rb);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&sm.p_half[i]);       // P of keys 0-63 is in place: P V may start
                 tmem_wait_ld();
                 chunk_exp<true>(ra, mk2, sl2, neg_ms, l2, pk);
                 tmem_st16(s_addr + 32, pk);
@@ -433,6 +441,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 chunk_exp<false>(rb, 0u, sl2, neg_ms, l2, pk);
                 tmem_st16(s_addr + 16, pk);
                 tmem_ld32(s_addr + 96, rb);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&sm.p_half[i]);       // P of keys 0-63 is in place: P V may start
                 tmem_wait_ld();
                 chunk_exp<false>(ra, 0u, sl2, neg_ms, l2, pk);
                 tmem_st16(s_addr + 32, pk);
