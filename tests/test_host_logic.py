@@ -36,6 +36,13 @@ def test_named_configs_have_the_stated_shapes():
     for p in (p2, p3, p4):
         lens = np.diff(p.cu_seqlens)
         assert lens.min() >= 16 and lens.sum() == p.n_main
+    # the shape of the paper's packed variable-length operator benchmark (Section 4.4):
+    # longest sequence 20,480 tokens, padded-to-longest size about 2.25x the real size
+    pv = W.varlen_ttt()
+    lens = np.diff(pv.cu_seqlens)
+    assert lens.max() == 20480 and pv.n_main == 73728 and pv.n_branch == 3 * 73728 and pv.kind == W.CHAIN
+    assert 2.1 < len(lens) * lens.max() / lens.sum() < 2.3
+    assert W.useful_pairs(pv) == 1871249408
 
 
 def test_generators_are_seeded_and_bf16_exact():
