@@ -87,8 +87,7 @@ __device__ __forceinline__ void chunk_pt(const uint32_t (&r)[32], uint32_t mk, f
 // dS^T of 32 query columns: P o (dP - dl[c]) as 16 packed bf16 pairs (invisible -> 0)
 template <bool MASKED>
 __device__ __forceinline__ void chunk_dst(const uint32_t (&r)[32], const uint32_t *pr, uint32_t mk,
-                                          const float *dl, uint32_t (&pk)[16]) {
-    const float4 *dl4 = reinterpret_cast<const float4 *>(dl);
+                                          const float4 *dl4, uint32_t (&pk)[16]) {
 #pragma unroll
     for (int e = 0; e < 32; e += 4) {
         const float4 dv = dl4[e >> 2];
@@ -511,6 +510,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&sm.a_done);
+            // delta of my first 32 columns goes into registers while this warp would wait anyway
+            // (phase B is on the critical chain and its shared-memory loads queue behind the SS MMAs)
+            float4 d0[8];
+#pragma unroll
+            for (int i4 = 0; i4 < 8; ++i4) d0[i4] = reinterpret_cast<const float4 *>(dl)[i4];
 
             // --- phase B: dS^T = P^T o (dP^T - delta[col]) -> shared memory (bf16)
             ok = mbar_wait(&sm.dp_full, t & 1, abort_flag);
@@ -522,14 +526,14 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                 tmem_ld32(x_addr, ra);
                 tmem_ld32(x_addr + 32, rb);
                 tmem_wait_ld();
-                if (masked) chunk_dst<true>(ra, &pr[0], mk0, dl, pk);
-                else chunk_dst<false>(ra, &pr[0], 0u, dl, pk);
+                if (masked) chunk_dst<true>(ra, &pr[0], mk0, d0, pk);
+                else chunk_dst<false>(ra, &pr[0], 0u, d0, pk);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch)
                     st_shared_v4(ds_row + (((uint32_t)ch ^ ds_xor) << 4), pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2],
                                  pk[4 * ch + 3]);
-                if (masked) chunk_dst<true>(rb, &pr[16], mk1, dl + 32, pk);
-                else chunk_dst<false>(rb, &pr[16], 0u, dl + 32, pk);
+                if (masked) chunk_dst<true>(rb, &pr[16], mk1, reinterpret_cast<const float4 *>(dl + 32), pk);
+                else chunk_dst<false>(rb, &pr[16], 0u, reinterpret_cast<const float4 *>(dl + 32), pk);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch)
                     st_shared_v4(ds_row + (((uint32_t)(ch + 4) ^ ds_xor) << 4), pk[4 * ch], pk[4 * ch + 1],
