@@ -276,7 +276,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
         }
     } else if (warp == 8) {
         // ================================================= MMA issuer
-        if (lane == 0 && T > 0) {
+        // The whole warp runs this code and an elected lane issues each MMA and commit: with
+        // warp-uniform control flow the descriptors stay in uniform registers, which halves what
+        // a tcgen05.mma costs its thread.  Every lane waits, and all agree on the outcome.
+        if (T > 0) {
             constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, 0);
             constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, 1);
             // low descriptor words (the issuing thread advances them with one add per MMA)
@@ -287,47 +290,47 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 const uint32_t k_km = kv_km0 + stage * kStageStep;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ss_lh(tmem + i * 128, q_km[i] + desc_step_kmajor(ks), k_km + desc_step_kmajor(ks), IDESC_QK, ks > 0);
+                    if (elect_one()) mma_ss_lh(tmem + i * 128, q_km[i] + desc_step_kmajor(ks), k_km + desc_step_kmajor(ks), IDESC_QK, ks > 0);
             };
             auto issue_pv = [&](int i, int stage, bool accumulate, int ks0) {   // K steps ks0 .. ks0 + 3
                 const uint32_t v_mn = kv_mn0 + stage * kStageStep;
 #pragma unroll
                 for (int ks = ks0; ks < ks0 + 4; ++ks)
-                    mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, v_mn + desc_step_mnmajor(ks), IDESC_PV,
+                    if (elect_one()) mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, v_mn + desc_step_mnmajor(ks), IDESC_PV,
                               accumulate || ks > 0);
             };
-            bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-            ok = ok && mbar_wait(&sm.kv_full[0], 0, abort_flag);
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full, 0, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(&sm.kv_full[0], 0, abort_flag));
             if (ok) {
                 tc_fence_after();
-                issue_qk(0, 0); tc_commit(&sm.s_full[0]);
-                issue_qk(1, 0); tc_commit(&sm.s_full[1]);
-                tc_commit(&sm.kv_empty[0]);
+                issue_qk(0, 0); if (elect_one()) tc_commit(&sm.s_full[0]);
+                issue_qk(1, 0); if (elect_one()) tc_commit(&sm.s_full[1]);
+                if (elect_one()) tc_commit(&sm.kv_empty[0]);
             }
             for (int j = 0; j < T && ok; ++j) {
                 const int it_v = 2 * j + 1, sv = it_v % kStages;
                 const int it_k = 2 * j + 2, sk = it_k % kStages;
                 for (int i = 0; i < 2 && ok; ++i) {
-                    ok = mbar_wait(&sm.p_half[i], j & 1, abort_flag);
-                    if (ok && i == 0) ok = mbar_wait(&sm.kv_full[sv], (it_v / kStages) & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.p_half[i], j & 1, abort_flag));
+                    if (ok && i == 0) ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full[sv], (it_v / kStages) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(i, sv, j > 0, 0);            // keys 0-63 while the softmax warps finish keys 64-127
-                    ok = mbar_wait(&sm.p_full[i], j & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.p_full[i], j & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(i, sv, true, 4);
-                    if (i == 1) tc_commit(&sm.kv_empty[sv]);
+                    if (i == 1) if (elect_one()) tc_commit(&sm.kv_empty[sv]);
                     if (j + 1 < T) {
                         if (i == 0) {
-                            ok = mbar_wait(&sm.kv_full[sk], (it_k / kStages) & 1, abort_flag);
+                            ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full[sk], (it_k / kStages) & 1, abort_flag));
                             if (!ok) break;
                             tc_fence_after();
                         }
-                        issue_qk(i, sk); tc_commit(&sm.s_full[i]);
-                        if (i == 1) tc_commit(&sm.kv_empty[sk]);
+                        issue_qk(i, sk); if (elect_one()) tc_commit(&sm.s_full[i]);
+                        if (i == 1) if (elect_one()) tc_commit(&sm.kv_empty[sk]);
                     } else {
-                        tc_commit(&sm.o_full[i]);
+                        if (elect_one()) tc_commit(&sm.o_full[i]);
                     }
                 }
             }
