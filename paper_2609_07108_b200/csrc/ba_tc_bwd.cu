@@ -202,7 +202,9 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
         }
     } else if (warp == 8) {
         // ================================================= MMA issuer
-        if (lane == 0 && T > 0) {
+        // the whole warp runs this code, an elected lane issues each MMA and commit (descriptors
+        // then stay in uniform registers); every lane waits and all agree on the outcome
+        if (T > 0) {
             constexpr uint32_t IDESC_KMAJ = idesc_bf16(128, 128, 0);  // S = Q K^T, dP = dO V^T
             constexpr uint32_t IDESC_MN = idesc_bf16(128, 128, 1);    // dQ += dS K
             // low descriptor words (the issuing thread advances them with one add per MMA)
@@ -214,48 +216,48 @@ tc_dq_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_constan
             auto issue_kmajor = [&](uint32_t d_tmem, uint32_t a_km, uint32_t b_km) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + desc_step_kmajor(ks), IDESC_KMAJ, ks > 0);
+                    if (elect_one()) mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + desc_step_kmajor(ks), IDESC_KMAJ, ks > 0);
             };
             auto issue_dq = [&](int i, uint32_t kmn, bool accumulate) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, kmn + desc_step_mnmajor(ks), IDESC_MN,
+                    if (elect_one()) mma_ts_lh(tmem + 256 + i * 128, tmem + i * 128 + ks * 8, kmn + desc_step_mnmajor(ks), IDESC_MN,
                               accumulate || ks > 0);
             };
-            bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-            ok = ok && mbar_wait(&sm.k_full[0], 0, abort_flag);
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full, 0, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(&sm.k_full[0], 0, abort_flag));
             if (ok) {
                 tc_fence_after();
-                issue_kmajor(tmem + 0, q_addr[0], k_km[0]); tc_commit(&sm.s_full[0]);
-                issue_kmajor(tmem + 128, q_addr[1], k_km[0]); tc_commit(&sm.s_full[1]);
+                issue_kmajor(tmem + 0, q_addr[0], k_km[0]); if (elect_one()) tc_commit(&sm.s_full[0]);
+                issue_kmajor(tmem + 128, q_addr[1], k_km[0]); if (elect_one()) tc_commit(&sm.s_full[1]);
             }
             for (int j = 0; j < T && ok; ++j) {
                 const int kb = j & 1;
                 for (int i = 0; i < 2 && ok; ++i) {
-                    ok = mbar_wait(&sm.a_done[i], j & 1, abort_flag);
-                    if (ok && i == 0) ok = mbar_wait(&sm.v_full, j & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.a_done[i], j & 1, abort_flag));
+                    if (ok && i == 0) ok = __all_sync(0xffffffffu, mbar_wait(&sm.v_full, j & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     issue_kmajor(tmem + i * 128, go_addr[i], v_km);
-                    tc_commit(&sm.dp_full[i]);
-                    if (i == 1) tc_commit(&sm.v_empty);
+                    if (elect_one()) tc_commit(&sm.dp_full[i]);
+                    if (i == 1) if (elect_one()) tc_commit(&sm.v_empty);
                 }
                 for (int i = 0; i < 2 && ok; ++i) {
-                    ok = mbar_wait(&sm.b_done[i], j & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.b_done[i], j & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     issue_dq(i, k_mn[kb], j > 0);
-                    if (i == 1) tc_commit(&sm.k_empty[kb]);
+                    if (i == 1) if (elect_one()) tc_commit(&sm.k_empty[kb]);
                     if (j + 1 < T) {
                         if (i == 0) {
-                            ok = mbar_wait(&sm.k_full[kb ^ 1], ((j + 1) >> 1) & 1, abort_flag);
+                            ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_full[kb ^ 1], ((j + 1) >> 1) & 1, abort_flag));
                             if (!ok) break;
                             tc_fence_after();
                         }
                         issue_kmajor(tmem + i * 128, q_addr[i], k_km[kb ^ 1]);
-                        tc_commit(&sm.s_full[i]);
+                        if (elect_one()) tc_commit(&sm.s_full[i]);
                     } else {
-                        tc_commit(&sm.dq_full[i]);
+                        if (elect_one()) tc_commit(&sm.dq_full[i]);
                     }
                 }
             }
@@ -631,7 +633,8 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
         }
     } else if (warp == 8) {
         // ================================================= MMA issuer
-        if (lane == 0 && n_iter > 0) {
+        // the whole warp runs this code, an elected lane issues each MMA and commit
+        if (n_iter > 0) {
             constexpr uint32_t IDESC_T = idesc_bf16(128, kSub, 0);   // 128 keys x 64 rows, K = d
             constexpr uint32_t IDESC_ACC = idesc_bf16(128, 128, 1);  // 128 keys x 128 d, K = 64 rows
             // low descriptor words (the issuing thread advances them with one add per MMA);
@@ -642,45 +645,45 @@ tc_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_const
             auto issue_t = [&](uint32_t d_tmem, uint32_t a_km, uint32_t b_km) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + (uint32_t)((ks >> 2) * 512 + (ks & 3) * 2),
+                    if (elect_one()) mma_ss_lh(d_tmem, a_km + desc_step_kmajor(ks), b_km + (uint32_t)((ks >> 2) * 512 + (ks & 3) * 2),
                               IDESC_T, ks > 0);
             };
             auto issue_acc = [&](uint32_t d_tmem, uint32_t a_tmem, uint32_t b_mn, bool accumulate) {
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    mma_ts_lh(d_tmem, a_tmem + ks * 8, b_mn + desc_step_mnmajor(ks), IDESC_ACC, accumulate || ks > 0);
+                    if (elect_one()) mma_ts_lh(d_tmem, a_tmem + ks * 8, b_mn + desc_step_mnmajor(ks), IDESC_ACC, accumulate || ks > 0);
             };
-            bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full, 0, abort_flag));
             for (int b = 0; b < 2 && ok; ++b) {
                 if (b >= n_iter) break;
-                ok = mbar_wait(&sm.q_full[b], 0, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full[b], 0, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 issue_t(tmem + 256 + b * 128, k_km, qs_km0 + b * kStageStep);                    // S^T = K Q^T
                 issue_t(tmem + 256 + b * 128 + 64, v_km, qs_km0 + b * kStageStep + kHalfStage);  // dP^T = V dO^T
-                tc_commit(&sm.sd_full[b]);
+                if (elect_one()) tc_commit(&sm.sd_full[b]);
             }
             for (int t = 0; t < n_iter && ok; ++t) {
                 const int b = t & 1;
                 const uint32_t stage_mn = qs_mn0 + (t % kQStages) * kStageStep;
-                ok = mbar_wait(&sm.pd_done[b], (t >> 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.pd_done[b], (t >> 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 issue_acc(tmem + 128, tmem + 256 + b * 128, stage_mn + kHalfStage, t > 0);   // dV += P^T dO
                 issue_acc(tmem + 0, tmem + 256 + b * 128 + 64, stage_mn, t > 0);             // dK += dS^T Q
-                tc_commit(&sm.q_empty[t % kQStages]);
+                if (elect_one()) tc_commit(&sm.q_empty[t % kQStages]);
                 const int t2 = t + 2;
                 if (t2 < n_iter) {
                     const uint32_t next_km = qs_km0 + (t2 % kQStages) * kStageStep;
-                    ok = mbar_wait(&sm.q_full[t2 % kQStages], (t2 / kQStages) & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full[t2 % kQStages], (t2 / kQStages) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     issue_t(tmem + 256 + b * 128, k_km, next_km);
                     issue_t(tmem + 256 + b * 128 + 64, v_km, next_km + kHalfStage);
-                    tc_commit(&sm.sd_full[b]);
+                    if (elect_one()) tc_commit(&sm.sd_full[b]);
                 }
             }
-            if (ok) tc_commit(&sm.acc_full);
+            if (ok) if (elect_one()) tc_commit(&sm.acc_full);
         }
     } else {
         // ================================================= P^T / dS^T warps + epilogue
