@@ -276,6 +276,12 @@ def run_step(rec, plan, t, cp, backward, fused=False):
     return o, lse, grads
 
 
+def use_fused_bwd(args, p, plan, ba):
+    if plan.impl != ba.IMPL_TC or args.bwd == "split":
+        return False
+    return args.bwd == "fused" or p.n_main >= 131072
+
+
 def run_ours(args):
     import torch
     from paper_2609_07108_b200 import binding as ba
@@ -314,7 +320,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    fused = args.bwd == "fused" and plan.impl == ba.IMPL_TC
+    fused = use_fused_bwd(args, p, plan, ba)
     for _ in range(args.warmup):
         run_step(rec, plan, t, cp, backward, fused=fused)
         if flush is not None:
@@ -481,7 +487,7 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     # forward: their copies run on side streams behind the forward / the backward.
     main = torch.cuda.current_stream()
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-    fused = args.bwd == "fused" and plan.impl == ba.IMPL_TC
+    fused = use_fused_bwd(args, p, plan, ba)
     for _ in range(steps):
         for k in names:
             if k != "d_o":
@@ -644,9 +650,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="auto", choices=["auto", *WORKLOADS])
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tc"])
-    ap.add_argument("--bwd", default="fused", choices=["split", "fused"],
-                    help="backward: dQ kernel + dK/dV kernel, or one kernel for all three (dQ summed "
-                         "with atomic adds)")
+    ap.add_argument("--bwd", default="auto", choices=["auto", "split", "fused"],
+                    help="backward: dQ kernel + dK/dV kernel, or one kernel for all three (dQ summed with "
+                         "atomic adds); auto = the one-kernel form from 131,072 tokens up (runs of seconds "
+                         "at the power cap, decided by the work done), the two-kernel form below")
     ap.add_argument("--branch-only", action="store_true",
                     help="q_main = NULL: only the branch tokens are queries (monolithic workloads)")
     ap.add_argument("--no-e2e", action="store_true")
