@@ -47,13 +47,39 @@ WORKLOADS = {
 }
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the launches of
-# one step) from a one-pass ncu capture of the full-size command; not measurable live.  The command
-# and the per-launch breakdown are in profiles/dram_traffic_config5_256k_zigzag.md.
-NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("config5_256k_zigzag", "tc_bwd_fused_kernel"): 11.36e9,
-    ("config5_256k_zigzag_fwd", "tc_fwd_kernel"): 5.68e9,
-}
+# DRAM traffic of the dominant kernels comes from profiles/dram_traffic.json: one ncu capture
+# per kernel on a small case (dram__bytes_read.sum + dram__bytes_write.sum of one launch),
+# stored with the hash of the kernel's source files at capture time.  It is scaled to this
+# workload's launches by the query rows a launch streams (Q, dO and the dQ accumulator rows
+# are what the kernel moves); if the sources have changed since the capture, traffic is null.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+CSRC = os.path.join(ROOT, "paper_2609_07108_b200", "csrc")
+
+
+def source_hash(files):
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(files):
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel_name, rows_per_launch):
+    """(bytes per launch scaled to `rows_per_launch`, description) or (None, reason)."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            table = json.load(f)
+    except (OSError, ValueError):
+        return None, "no capture on file"
+    e = table.get(kernel_name)
+    if not e:
+        return None, "no capture on file"
+    if source_hash(e["source_files"]) != e["source_hash"]:
+        return None, "kernel source changed since the capture"
+    scaled = e["dram_bytes_per_launch"] * rows_per_launch / e["query_rows_per_launch"]
+    return scaled, (f"ncu one launch on {e['case']} ({e['dram_bytes_per_launch'] / 1e6:.0f} MB for "
+                    f"{e['query_rows_per_launch']} query rows) scaled by query rows; commit {e['commit']}")
 
 
 def useful_flops(p, backward=True, branch_only=False):
@@ -179,7 +205,8 @@ class Recorder:
         self.events = []           # (kind, start, end)
         self.launches = 0
         self.enabled = False
-        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL", "STAGE_ALL", "STAGE_ALL_FUSED", "IMPL_TC"):
+        for name in ("PART_MAIN", "PART_BRANCH", "PART_ALL", "STAGE_ALL", "STAGE_ALL_FUSED", "STAGE_PREP", "STAGE_DQ",
+                     "STAGE_DKDV", "STAGE_FUSED", "IMPL_TC"):
             setattr(self, name, getattr(ba, name))
 
     def _wrap(self, kind, n_launch, fn, *a, **k):
@@ -207,21 +234,27 @@ class Recorder:
         return self._wrap("lse_merge", 1, self.ba.lse_merge, *a, **k)
 
     def branch_attn_bwd(self, plan, q_main, *a, **k):
-        # the three stages of one backward call, bracketed separately:
-        # preprocess (delta of main rows, of branch rows), dQ kernel, dK/dV kernel
+        # every stage of a backward call is bracketed separately: preprocess (one launch for the
+        # main and the branch rows), dQ kernel, dK/dV kernel -- or the one fused kernel
         ba = self.ba
         k = dict(k)
-        fused = k.pop("stages", ba.STAGE_ALL) == ba.STAGE_ALL_FUSED
+        stages = k.pop("stages", ba.STAGE_ALL)
+        acc = k.get("accumulate", False)
+        fused_extra = 0 if acc else (2 if q_main is not None else 1)   # conversion of the fp32 dQ accumulators
+        single = {ba.STAGE_PREP: ("bwd_prep", 1), ba.STAGE_DQ: ("bwd_dq", 1), ba.STAGE_DKDV: ("bwd_dkdv", 1),
+                  ba.STAGE_FUSED: ("bwd_fused", 1 + fused_extra)}
+        if stages in single:
+            kind, n_l = single[stages]
+            return self._wrap(kind, n_l, ba.branch_attn_bwd, plan, q_main, *a, stages=stages, **k)
+        fused = stages == ba.STAGE_ALL_FUSED
         # gradients in the input dtype through the one-kernel backward: all stages share the larger workspace
-        prep_kw = {"fused_scratch": True} if fused and not k.get("accumulate", False) else {}
-        out = self._wrap("bwd_prep", 2 if q_main is not None else 1, ba.branch_attn_bwd, plan, q_main, *a,
-                         stages=ba.STAGE_PREP, **prep_kw, **k)
+        prep_kw = {"fused_scratch": True} if fused and not acc else {}
+        out = self._wrap("bwd_prep", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_PREP, **prep_kw, **k)
         k2 = dict(k)
         k2["grads"] = out
         if fused:   # one kernel for dQ, dK and dV
-            # (without accumulate: plus the conversion of the dQ accumulators of main and branch rows)
-            n_l = 1 if k.get("accumulate", False) else (3 if q_main is not None else 2)
-            return self._wrap("bwd_fused", n_l, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_FUSED, **k2)
+            return self._wrap("bwd_fused", 1 + fused_extra, ba.branch_attn_bwd, plan, q_main, *a,
+                              stages=ba.STAGE_FUSED, **k2)
         self._wrap("bwd_dq", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DQ, **k2)
         return self._wrap("bwd_dkdv", 1, ba.branch_attn_bwd, plan, q_main, *a, stages=ba.STAGE_DKDV, **k2)
 
@@ -256,7 +289,7 @@ def run_fwd(rec, plan, t, cp):
     from paper_2609_07108_b200 import zigzag
     if cp:
         o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp,
-                                   out=t.get("_o"), lse=t.get("_lse"))
+                                   out=t.get("_o"), lse=t.get("_lse"), ws=t.get("_ws"))
         return o, lse
     return rec.branch_attn_fwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], out=t.get("_o"), lse=t.get("_lse"))
 
@@ -265,7 +298,7 @@ def run_bwd(rec, plan, t, cp, o, lse, fused=False):
     from paper_2609_07108_b200 import zigzag
     if cp:
         return zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp,
-                               fused=fused)
+                               fused=fused, ws=t.get("_ws"))
     return rec.branch_attn_bwd(plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"],
                                grads=t.get("_grads"), stages=rec.STAGE_ALL_FUSED if fused else rec.STAGE_ALL)
 
@@ -298,6 +331,17 @@ def run_ours(args):
     p = W.CONFIGS[cfg](shrink) if cfg != 1 else W.config1()
     impl = {"auto": ba.IMPL_AUTO, "simt": ba.IMPL_SIMT, "tc": ba.IMPL_TC}[args.kernels]
     plan = ba.Plan(p, device=device, impl=impl)
+    # metadata builder, timed on its own (it is reused by the forward, the backward and, in a
+    # model, every layer): host wall clock around ba_plan_create incl. its stream synchronisations
+    plan_times = []
+    for _ in range(3):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        extra = ba.Plan(p, device=device, impl=impl)
+        torch.cuda.synchronize()
+        plan_times.append((time.perf_counter() - t0) * 1e3)
+        extra.close()
+    plan_ms = statistics.median(plan_times)
     branch_only = bool(args.branch_only)
     if branch_only and cp:
         raise SystemExit("--branch-only applies to the monolithic workloads")
@@ -305,9 +349,18 @@ def run_ours(args):
     t = make_device_inputs(p, torch, device)
     if branch_only:
         t["q_main"] = None   # draft-only form: main K/V are keys, only branch tokens are queries
-    if not cp:
-        t["_o"] = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
-        t["_lse"] = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=device)
+    # outputs and (zigzag) the fp32 accumulators are allocated once, outside the steps
+    t["_o"] = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
+    t["_lse"] = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=device)
+    if cp:
+        from paper_2609_07108_b200 import zigzag
+        t["_ws"] = zigzag.Workspace(ba, plan, cp, backward=backward)
+    elif backward:
+        t["_grads"] = (torch.empty((p.n_main, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
+                       if not branch_only else None,
+                       torch.empty((p.n_branch, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device),
+                       torch.empty((p.rows, p.h_kv, p.head_dim), dtype=plan.torch_dtype, device=device),
+                       torch.empty((p.rows, p.h_kv, p.head_dim), dtype=plan.torch_dtype, device=device))
     rec = Recorder(ba, p)
     in_bytes = sum(t[k].numel() * t[k].element_size() for k in ("q_main", "q_branch", "k", "v", "d_o")
                    if t[k] is not None)
@@ -338,7 +391,7 @@ def run_ours(args):
         s = torch.cuda.Event(enable_timing=True)
         e = torch.cuda.Event(enable_timing=True)
         s.record()
-        run_step(rec, plan, t, cp, backward, fused=fused)
+        last = run_step(rec, plan, t, cp, backward, fused=fused)
         e.record()
         step_ms.append((s, e))
     barrier()
@@ -348,6 +401,13 @@ def run_ours(args):
     value, total_ms = aggregate_throughput(dist, flops * args.steps, local_ms, device)
     totals = rec.totals()
     launches = rec.launches
+
+    # ---- CPU baseline (the oracle on a bounded sample of the same inputs) and the GPU's error
+    # against it on those rows; before the end-to-end run, which overwrites inputs and outputs
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(p, seconds_target=15.0, backward=backward,
+                           gpu=None if branch_only else (t, last))
 
     # ---- end to end through the API with HOST buffers (pinned), copies timed
     e2e = None
@@ -371,11 +431,16 @@ def run_ours(args):
             kflops = pairs * p.head_dim * p.h_q * share * args.steps
             achieved = kflops / (ms * 1e-3) / 1e12
             long_step = total_ms / args.steps > 1000.0
+            # query rows (row, head) one launch streams on average, for scaling the ncu traffic capture
+            rows_per_launch = query_rows_streamed(p, cp, kind) * args.steps / max(calls, 1)
+            traffic, traffic_src = ncu_traffic(kernel_name, rows_per_launch)
+            if traffic is not None:
+                traffic = round(traffic)
             peak = peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"]
             roof = {"bound": "tensor", "kernel": kernel_name, "flop_per_pair_head": share * p.head_dim,
                     "achieved": round(achieved, 2), "peak": peak,
                     "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
-                    "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((name, kernel_name)),
+                    "traffic": traffic, "traffic_source": traffic_src,
                     "peak_source": f"{peaks['_source']} {'sustained' if long_step else 'burst'} bf16",
                     "launches": calls, "avg_launch_ms": round(ms / calls, 4),
                     "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
@@ -384,9 +449,6 @@ def run_ours(args):
             roof = {"bound": "hbm", "kernel": kind, "achieved": None, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": None, "traffic": None}
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(p, seconds_target=15.0)
 
     if rank == 0:
         line = {
@@ -413,6 +475,7 @@ def run_ours(args):
                              "datasheet": round(value / world / DATASHEET_BF16_TFLOPS, 4),
                              "source": peaks["_source"]},
             "kernel_ms": {k: round(v[0] / args.steps, 3) for k, v in totals.items()},
+            "plan_ms": round(plan_ms, 3),
             "gpu_launches": launches,
             "clocks": clocks,
             "e2e": e2e,
@@ -532,15 +595,46 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
 # CPU baseline = the oracle, as it stands, on a bounded sample
 # ----------------------------------------------------------------------------
 
-def oracle_sample(p, n_rows, seed=0):
+def query_rows_streamed(p, cp, kind):
+    """Query rows one step's launches of `kind` stream in total (a row counts once per launch
+    that walks it): every row once for a monolithic call, once per (q chunk, kv chunk) block of
+    the emulated ring."""
+    if not cp:
+        return p.rows
+    from paper_2609_07108_b200 import zigzag
+    total = 0
+    offs = p.branch_offsets.astype(np.int64)
+    for b in zigzag.schedule(p, cp):
+        total += (b.qm[1] - b.qm[0]) + int(offs[b.br[1]] - offs[b.br[0]])
+    return total
+
+
+def oracle_sample(p, n_rows, seed=0, gpu_inputs=None):
     """Rows sampled uniformly from the workload (main and branch rows), one KV
-    group (h_q/h_kv query heads).  Returns the inputs and the sampled pairs."""
+    group (h_q/h_kv query heads).  Returns the inputs and the sampled rows.  With
+    `gpu_inputs` (the benchmark's device tensors) the values are those the GPU ran
+    on, so that the oracle's results can be compared with the GPU's."""
     import copy
     rng = np.random.default_rng(seed)
     rows = np.sort(rng.choice(p.rows, size=min(n_rows, p.rows), replace=False)).astype(np.int64)
     p1 = copy.copy(p)
     p1.h_q, p1.h_kv = p.h_q // p.h_kv, 1
     d = p.head_dim
+    if gpu_inputs is not None:
+        import torch
+        t = gpu_inputs
+        n, g = p.n_main, p1.h_q
+        dev = t["k"].device
+        is_b = rows >= n
+        q = np.empty((len(rows), g, d), dtype=np.float32)
+        if (~is_b).any():
+            q[~is_b] = t["q_main"][torch.from_numpy(rows[~is_b]).to(dev)][:, :g].float().cpu().numpy()
+        if is_b.any():
+            q[is_b] = t["q_branch"][torch.from_numpy(rows[is_b] - n).to(dev)][:, :g].float().cpu().numpy()
+        k = t["k"][:, :1].float().cpu().numpy()
+        v = t["v"][:, :1].float().cpu().numpy()
+        go = t["d_o"][torch.from_numpy(rows).to(dev)][:, :g].float().cpu().numpy()
+        return p1, rows, q, k, v, go
     q = W.round_to_bf16(rng.standard_normal((len(rows), p1.h_q, d), dtype=np.float32) * 0.5)
     k = W.round_to_bf16(rng.standard_normal((p.rows, 1, d), dtype=np.float32) * 0.5)
     v = W.round_to_bf16(rng.standard_normal((p.rows, 1, d), dtype=np.float32) * 0.5)
@@ -574,39 +668,77 @@ def sample_pairs(oracle, p1, rows):
     return int(total)
 
 
-def time_oracle(p, n_rows, backward=True):
+def time_oracle(p, n_rows, backward=True, gpu_inputs=None, keep=False):
     from oracle import oracle
     oracle.build()
-    p1, rows, q, k, v, go = oracle_sample(p, n_rows)
+    p1, rows, q, k, v, go = oracle_sample(p, n_rows, gpu_inputs=gpu_inputs)
     pairs = sample_pairs(oracle, p1, rows)
     t0 = time.perf_counter()
+    res = {}
     if backward:
-        oracle.backward(p1, q, k, v, go, rows=rows)       # runs the forward inside
+        res["dq"] = oracle.backward(p1, q, k, v, go, rows=rows)[0]       # runs the forward inside
     else:
-        oracle.forward(p1, q, k, v, rows=rows)
+        res["o"], res["lse"] = oracle.forward(p1, q, k, v, rows=rows)
     dt = time.perf_counter() - t0
+    if keep and backward:                                                # untimed: O and LSE for the comparison
+        res["o"], res["lse"] = oracle.forward(p1, q, k, v, rows=rows)
     fl = pairs * 4 * p.head_dim * p1.h_q * (3.5 if backward else 1.0)
-    return fl / dt / 1e12, dt, len(rows), pairs, p1.h_q
+    return fl / dt / 1e12, dt, len(rows), pairs, p1.h_q, (rows, res) if keep else None
 
 
 def sized_rows(p, seconds_target, backward):
     """Sample size whose oracle run takes about `seconds_target` (found by doubling)."""
     n_rows, dt = 8, 0.0
     while n_rows < p.rows:
-        _, dt, _, _, _ = time_oracle(p, n_rows, backward)
+        _, dt, _, _, _, _ = time_oracle(p, n_rows, backward)
         if dt >= seconds_target / 4:
             break
         n_rows *= 4
     return int(max(8, min(p.rows, n_rows * seconds_target / max(dt, 1e-3))))
 
 
-def cpu_baseline(p, seconds_target=15.0, backward=True):
+def gpu_vs_oracle(p, rows, res, gpu):
+    """max abs and rel-RMS error of the GPU's O, LSE and dQ of the last timed step against the
+    oracle on the CPU-baseline sample rows (first KV group)."""
+    import torch
+    t, last = gpu
+    o, lse, grads = last
+    g = p.h_q // p.h_kv
+    n = p.n_main
+    dev = o.device
+    rows_t = torch.from_numpy(rows).to(dev)
+
+    def metrics(got, want):
+        err = got.astype(np.float64) - want
+        den = float(np.sqrt(np.mean(want * want)))
+        return {"max_abs": float(f"{np.abs(err).max():.3e}"),
+                "rel_rms": float(f"{np.sqrt(np.mean(err * err)) / den:.3e}") if den > 0 else None}
+
+    out = {"rows": int(len(rows)), "heads": g}
+    out["O"] = metrics(o[rows_t][:, :g].float().cpu().numpy(), res["o"])
+    out["LSE"] = metrics(lse[rows_t][:, :g].float().cpu().numpy(), res["lse"])
+    if grads is not None and "dq" in res:
+        is_b = rows >= n
+        dq = np.empty((len(rows), g, p.head_dim), dtype=np.float32)
+        if (~is_b).any():
+            dq[~is_b] = grads[0][torch.from_numpy(rows[~is_b]).to(dev)][:, :g].float().cpu().numpy()
+        if is_b.any():
+            dq[is_b] = grads[1][torch.from_numpy(rows[is_b] - n).to(dev)][:, :g].float().cpu().numpy()
+        out["dQ"] = metrics(dq, res["dq"])
+    return out
+
+
+def cpu_baseline(p, seconds_target=15.0, backward=True, gpu=None):
     cores = len(os.sched_getaffinity(0))
     n_rows = sized_rows(p, seconds_target, backward)
-    val, dt, nr, pairs, hq = time_oracle(p, n_rows, backward)
-    return {"value": float(f"{val:.6g}"), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{nr} uniformly sampled query rows x {hq} query heads of one KV group, "
-                      f"fwd{'+bwd' if backward else ''}, {pairs} visible pairs per head, {dt:.1f} s"}
+    val, dt, nr, pairs, hq, kept = time_oracle(p, n_rows, backward, gpu_inputs=gpu[0] if gpu else None,
+                                               keep=gpu is not None)
+    out = {"value": float(f"{val:.6g}"), "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"{nr} uniformly sampled query rows x {hq} query heads of one KV group, "
+                     f"fwd{'+bwd' if backward else ''}, {pairs} visible pairs per head, {dt:.1f} s"}
+    if kept is not None:
+        out["gpu_vs_oracle"] = gpu_vs_oracle(p, kept[0], kept[1], gpu)
+    return out
 
 
 def run_reference(args):
@@ -622,7 +754,7 @@ def run_reference(args):
         time_oracle(p, 8, backward)
     vals, secs = [], []
     for _ in range(args.steps):
-        val, dt, nr, pairs, hq = time_oracle(p, n_rows, backward)
+        val, dt, nr, pairs, hq, _ = time_oracle(p, n_rows, backward)
         vals.append(val)
         secs.append(dt)
     value = sum(vals) / len(vals)

@@ -72,7 +72,8 @@ typedef struct ba_problem {
     int32_t impl;                  /* BA_IMPL_* */
     const int32_t *cu_seqlens;     /* device [B+1], cu[0] = 0, cu[B] = N, non-decreasing */
     const int32_t *anchor_idx;     /* device [A], global packed index in [0, N), non-decreasing */
-    const int32_t *branch_offsets; /* device [A+1] token offsets (0 .. M), or NULL with uniform_len */
+    const int32_t *branch_offsets; /* device [A+1] token offsets (0 .. M); may be NULL with
+                                      uniform_len > 0 or with A = 0 (it is not read then) */
     const int32_t *parent;         /* device [M], BA_MASK_TREE only: branch-local parent index,
                                       -1 = root, parent[i] < i */
 } ba_problem_t;
@@ -239,6 +240,8 @@ int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main, const void
  * that loads the library holds that much memory until the process exits.
  *   - Arguments are those of branch_attn_bwd without workspace / ws_bytes; the
  *     caller still owns all inputs and outputs.
+ *   - The size limit is checked first: a problem beyond it gets BA_EWORKSPACE
+ *     even for a call whose ranges are empty (where branch_attn_bwd returns BA_OK).
  *   - Limit: ba_workspace_bytes(plan, BA_OP_BWD) must not exceed
  *     BA_STATIC_SCRATCH_BYTES (8 MiB: 2 * h_q * (N + M + 128, rounded up to 64)
  *     floats, e.g. 32 query heads and up to 32,640 rows); larger problems get

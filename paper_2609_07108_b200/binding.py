@@ -105,6 +105,33 @@ def _p(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+def _expect(name, t, shape, dtype, device, optional=False):
+    """A tensor handed to the library must be exactly what the kernels and tensor
+    maps assume: on the plan's device, contiguous, of the stated dtype and shape.
+    (The library sees only a raw pointer; a strided view or a wrong dtype would
+    make it read or write outside the allocation.)"""
+    if t is None:
+        if optional:
+            return
+        raise ValueError(f"{name}: tensor required")
+    if not t.is_cuda or (device is not None and t.device != device):
+        raise ValueError(f"{name}: on {t.device}, expected {device}")
+    if t.dtype != dtype:
+        raise ValueError(f"{name}: dtype {t.dtype}, expected {dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: shape {tuple(t.shape)}, expected {tuple(shape)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: not contiguous")
+
+
+def _expect_inputs(plan, q_main, q_branch, k, v, q_main_optional=True):
+    p, dt, dev = plan.problem, plan.torch_dtype, plan.device
+    _expect("q_main", q_main, (p.n_main, p.h_q, p.head_dim), dt, dev, optional=q_main_optional)
+    _expect("q_branch", q_branch, (p.n_branch, p.h_q, p.head_dim), dt, dev, optional=p.n_branch == 0)
+    _expect("k", k, (p.rows, p.h_kv, p.head_dim), dt, dev)
+    _expect("v", v, (p.rows, p.h_kv, p.head_dim), dt, dev)
+
+
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
@@ -129,6 +156,8 @@ class Plan:
         lib = _lib()
         self.problem = problem
         self.device = torch.device(device)
+        if self.device.type == "cuda" and self.device.index is None:
+            self.device = torch.device("cuda", torch.cuda.current_device())
         self.dtype_code, self.torch_dtype = _DT[problem.dtype]
         offs = np.asarray(problem.branch_offsets, dtype=np.int64)
         lens = np.diff(offs)
@@ -141,7 +170,7 @@ class Plan:
                           problem.h_q, problem.h_kv, problem.head_dim, self.dtype_code,
                           float(problem.scale), int(problem.kind), uniform, impl,
                           self._cu.data_ptr(), self._anchor.data_ptr() if len(self._anchor) else None,
-                          self._offs.data_ptr(),
+                          self._offs.data_ptr() if problem.num_branches else None,   # A = 0: no branch arrays
                           self._parent.data_ptr() if self._parent is not None and len(self._parent) else None)
         nbytes = lib.ba_plan_bytes(C.byref(self.c))
         if nbytes == 0:
@@ -198,6 +227,9 @@ def branch_attn_fwd(plan, q_main, q_branch, k, v, out=None, lse=None):
         out = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=plan.device)
     if lse is None:
         lse = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=plan.device)
+    _expect_inputs(plan, q_main, q_branch, k, v)
+    _expect("out", out, (p.rows, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("lse", lse, (p.rows, p.h_q), torch.float32, plan.device)
     ws = plan.workspace(OP_FWD)
     rc = _lib().branch_attn_fwd(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(out), _p(lse),
                                 _p(ws), ws.numel(), _stream())
@@ -215,6 +247,9 @@ def branch_attn_fwd_partial(plan, q_main, q_branch, k, v, qm_range, br_range, kv
         out = torch.empty((rows, p.h_q, p.head_dim), dtype=torch.float32, device=plan.device)
     if lse is None:
         lse = torch.empty((rows, p.h_q), dtype=torch.float32, device=plan.device)
+    _expect_inputs(plan, q_main, q_branch, k, v)
+    _expect("out", out, (rows, p.h_q, p.head_dim), torch.float32, plan.device)
+    _expect("lse", lse, (rows, p.h_q), torch.float32, plan.device)
     ws = plan.workspace(OP_FWD)
     rc = _lib().branch_attn_fwd_partial(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v),
                                         qm_range[0], qm_range[1], br_range[0], br_range[1],
@@ -226,6 +261,12 @@ def branch_attn_fwd_partial(plan, q_main, q_branch, k, v, qm_range, br_range, kv
 
 def branch_attn_fwd_partial_merge(plan, q_main, q_branch, k, v, qm_range, br_range, kv_range, parts, acc_o, acc_lse):
     """Partial forward whose epilogue merges into the compact fp32 (acc_o, acc_lse) in place."""
+    p = plan.problem
+    t0, t1 = plan.token_range(*br_range)
+    rows = (qm_range[1] - qm_range[0]) + (t1 - t0)
+    _expect_inputs(plan, q_main, q_branch, k, v)
+    _expect("acc_o", acc_o, (rows, p.h_q, p.head_dim), torch.float32, plan.device)
+    _expect("acc_lse", acc_lse, (rows, p.h_q), torch.float32, plan.device)
     ws = plan.workspace(OP_FWD)
     rc = _lib().branch_attn_fwd_partial_merge(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v),
                                               qm_range[0], qm_range[1], br_range[0], br_range[1],
@@ -243,11 +284,33 @@ def lse_merge(o_a, lse_a, o_b, lse_b, out=None, lse_out=None, out_dtype=torch.fl
         out = torch.empty(o_a.shape, dtype=out_dtype, device=o_a.device)
     if lse_out is None:
         lse_out = torch.empty_like(lse_a)
+    dev = o_a.device
+    _expect("o_a", o_a, None, torch.float32, dev)
+    _expect("o_b", o_b, o_a.shape, torch.float32, dev)
+    _expect("lse_a", lse_a, o_a.shape[:-1], torch.float32, dev)
+    _expect("lse_b", lse_b, o_a.shape[:-1], torch.float32, dev)
+    _expect("out", out, o_a.shape, out.dtype, dev)
+    _expect("lse_out", lse_out, o_a.shape[:-1], torch.float32, dev)
+    if out.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"out: dtype {out.dtype} not supported")
     code = BA_BF16 if out.dtype == torch.bfloat16 else BA_FP32
     rc = _lib().lse_merge(items, d, _p(o_a), _p(lse_a), _p(o_b), _p(lse_b), _p(out), code,
                           _p(lse_out), _stream())
     _check(rc, "lse_merge")
     return out, lse_out
+
+
+def _expect_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, accumulate, grads):
+    p, dt, dev = plan.problem, plan.torch_dtype, plan.device
+    _expect_inputs(plan, q_main, q_branch, k, v)
+    _expect("o", o, (p.rows, p.h_q, p.head_dim), dt, dev)
+    _expect("lse", lse, (p.rows, p.h_q), torch.float32, dev)
+    _expect("d_o", d_o, (p.rows, p.h_q, p.head_dim), dt, dev)
+    gdt = torch.float32 if accumulate else dt
+    _expect("dQ_main", grads[0], (p.n_main, p.h_q, p.head_dim), gdt, dev, optional=q_main is None)
+    _expect("dQ_branch", grads[1], (p.n_branch, p.h_q, p.head_dim), gdt, dev, optional=p.n_branch == 0)
+    _expect("dK", grads[2], (p.rows, p.h_kv, p.head_dim), gdt, dev)
+    _expect("dV", grads[3], (p.rows, p.h_kv, p.head_dim), gdt, dev)
 
 
 def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br_range=None,
@@ -269,6 +332,7 @@ def branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=None, br
                  mk((p.n_branch, p.h_q, p.head_dim), dtype=dt, device=plan.device),
                  mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device),
                  mk((p.rows, p.h_kv, p.head_dim), dtype=dt, device=plan.device))
+    _expect_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, accumulate, grads)
     # every stage of one backward must see the same workspace: once a plan has been
     # used for the one-kernel backward with gradients in the input dtype (which keeps
     # an fp32 dQ accumulator in the workspace), all its backward calls use that buffer
@@ -303,6 +367,7 @@ def branch_attn_bwd_static(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=N
     kv_range = (0, p.n_main) if kv_range is None else kv_range
     if grads is None:
         raise ValueError("branch_attn_bwd_static writes into caller-provided gradient tensors")
+    _expect_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, accumulate, grads)
     rc = _lib().branch_attn_bwd_static(plan.handle, _p(q_main), _p(q_branch), _p(k), _p(v), _p(o), _p(lse),
                                        _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1],
                                        kv_range[0], kv_range[1], parts, 1 if accumulate else 0,
@@ -314,6 +379,10 @@ def branch_attn_bwd_static(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=N
 def ba_finalize_grads(src, dst=None, dtype=torch.bfloat16):
     if dst is None:
         dst = torch.empty(src.shape, dtype=dtype, device=src.device)
+    _expect("src", src, None, torch.float32, src.device)
+    _expect("dst", dst, src.shape, dst.dtype, src.device)
+    if dst.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"dst: dtype {dst.dtype} not supported")
     code = BA_BF16 if dst.dtype == torch.bfloat16 else BA_FP32
     rc = _lib().ba_finalize_grads(_p(src), _p(dst), src.numel(), code, _stream())
     _check(rc, "ba_finalize_grads")

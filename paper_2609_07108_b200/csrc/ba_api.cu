@@ -141,13 +141,10 @@ extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main,
     const int64_t rp = plan->row_pitch;
     const int64_t n = plan->prob.n_main;
     const int hq = plan->prob.h_q, d = plan->prob.head_dim, dt = plan->prob.dtype;
-    if (stages & BA_STAGE_PREP) {
-        if (has_main_q &&
-            (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, r.qm_begin, r.qm_end, hq, d, dt, st)) != BA_OK)
-            return rc;
-        if (has_branch_q &&
-            (rc = ba_delta(O, dO, LSE, delta, nlse2, rp, n + r.tok_begin, n + r.tok_end, hq, d, dt, st)) != BA_OK)
-            return rc;
+    if (stages & BA_STAGE_PREP) {   // main rows and branch rows of the call in one launch
+        const int64_t ma = has_main_q ? r.qm_begin : 0, mb = has_main_q ? r.qm_end : 0;
+        const int64_t ba_ = has_branch_q ? n + r.tok_begin : 0, bb = has_branch_q ? n + r.tok_end : 0;
+        if ((rc = ba_delta(O, dO, LSE, delta, nlse2, rp, ma, mb, ba_, bb, hq, d, dt, st)) != BA_OK) return rc;
     }
     if (!(stages & (BA_STAGE_DQ | BA_STAGE_DKDV | BA_STAGE_FUSED))) return BA_OK;
     const void *qm = has_main_q ? q_main : nullptr;

@@ -87,7 +87,8 @@ bool ba_tc_supported(const ba_problem_t *p);
 // Elementwise (ba_elementwise.cu)
 // Backward preprocess into head-major scratch [h_q, row_pitch]:
 //   delta_t[h, r] = <dO[r, h], O[r, h]>,  nlse2_t[h, r] = -LSE[r, h] * log2(e)
+// for two row segments [row_a_begin, row_a_end) and [row_b_begin, row_b_end) (either may be empty)
 int ba_delta(const void *o, const void *d_o, const float *lse, float *delta_t, float *nlse2_t,
-             int64_t row_pitch, int64_t row_begin, int64_t row_end, int h_q, int d, int dtype,
-             cudaStream_t st);
+             int64_t row_pitch, int64_t row_a_begin, int64_t row_a_end, int64_t row_b_begin,
+             int64_t row_b_end, int h_q, int d, int dtype, cudaStream_t st);
 static inline int64_t ba_row_pitch(int64_t rows) { return (rows + 128 + 63) / 64 * 64; }

@@ -31,7 +31,7 @@ __device__ __forceinline__ uint2 pack_bf16x4(float4 x) {
 // warp so that in-place updates (O_out == O_a, LSE_out == LSE_a) are safe.
 template <int LPI, bool OUT_BF16>
 __global__ void __launch_bounds__(kThreads)
-lse_merge_kernel(int64_t items, const float4 *__restrict__ oa, const float *lse_a,
+lse_merge_kernel(int64_t items, const float4 *oa, const float *lse_a,   // may alias o_out / lse_out: no __restrict__
                  const float4 *__restrict__ ob, const float *__restrict__ lse_b,
                  void *o_out, float *lse_out) {
     constexpr int IPW = 32 / LPI;  // items per warp
@@ -95,12 +95,14 @@ int launch_merge(int lpi, int64_t items, const float *oa, const float *la, const
 }
 
 // delta_t[h, r] = sum_d dO[r, h, d] * O[r, h, d] and nlse2_t[h, r] = -LSE[r, h] log2(e),
-// both head-major with `pitch` rows per head; one 16-byte chunk per lane.
+// both head-major with `pitch` rows per head; one 16-byte chunk per lane.  The rows are
+// two segments handled by one launch: [row_a, row_a + items_a / h_q), then rows from row_b
+// (the main query rows and the branch rows of one call).
 template <typename T, int LPI>
 __global__ void __launch_bounds__(kThreads)
-delta_kernel(int64_t items, const uint4 *__restrict__ o, const uint4 *__restrict__ d_o,
+delta_kernel(int64_t items, int64_t items_a, const uint4 *__restrict__ o, const uint4 *__restrict__ d_o,
              const float *__restrict__ lse, float *__restrict__ delta_t, float *__restrict__ nlse2_t,
-             int64_t row_begin, int h_q, int64_t pitch) {
+             int64_t row_a, int64_t row_b, int h_q, int64_t pitch) {
     constexpr int IPW = 32 / LPI;
     const int lane = threadIdx.x & 31;
     const int sub = lane % LPI;
@@ -109,8 +111,14 @@ delta_kernel(int64_t items, const uint4 *__restrict__ o, const uint4 *__restrict
     for (int64_t base = warp * IPW; base < items; base += warps * IPW) {
         const int64_t i = base + lane / LPI;
         float acc = 0.f;
+        int64_t r = 0;
+        int h = 0;
         if (i < items) {
-            const uint4 x = o[i * LPI + sub], y = d_o[i * LPI + sub];
+            const int64_t j = i < items_a ? i : i - items_a;
+            r = (i < items_a ? row_a : row_b) + j / h_q;
+            h = (int)(j % h_q);
+            const int64_t e = (r * h_q + h) * LPI + sub;
+            const uint4 x = o[e], y = d_o[e];
             if (sizeof(T) == 4) {
                 const float *xf = reinterpret_cast<const float *>(&x);
                 const float *yf = reinterpret_cast<const float *>(&y);
@@ -129,8 +137,6 @@ delta_kernel(int64_t items, const uint4 *__restrict__ o, const uint4 *__restrict
 #pragma unroll
         for (int off = LPI / 2; off; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         if (i < items && sub == 0) {
-            const int64_t r = row_begin + i / h_q;
-            const int h = (int)(i % h_q);
             delta_t[h * pitch + r] = acc;
             nlse2_t[h * pitch + r] = -lse[r * h_q + h] * 1.4426950408889634f;
         }
@@ -177,18 +183,19 @@ extern "C" int lse_merge(int64_t rows_heads, int d, const float *O_a, const floa
 }
 
 int ba_delta(const void *o, const void *d_o, const float *lse, float *delta_t, float *nlse2_t,
-             int64_t row_pitch, int64_t row_begin, int64_t row_end, int h_q, int d, int dtype,
-             cudaStream_t st) {
-    const int64_t items = (row_end - row_begin) * h_q;
+             int64_t row_pitch, int64_t row_a_begin, int64_t row_a_end, int64_t row_b_begin,
+             int64_t row_b_end, int h_q, int d, int dtype, cudaStream_t st) {
+    const int64_t items_a = row_a_end > row_a_begin ? (row_a_end - row_a_begin) * h_q : 0;
+    const int64_t items_b = row_b_end > row_b_begin ? (row_b_end - row_b_begin) * h_q : 0;
+    const int64_t items = items_a + items_b;
     if (items <= 0) return BA_OK;
     const size_t esz = dtype == BA_FP32 ? 4 : 2;
-    const uint4 *op = (const uint4 *)((const char *)o + (size_t)row_begin * h_q * d * esz);
-    const uint4 *gp = (const uint4 *)((const char *)d_o + (size_t)row_begin * h_q * d * esz);
+    const uint4 *op = (const uint4 *)o, *gp = (const uint4 *)d_o;
     const int lpi = (int)(d * esz / 16);
     const int grid = stream_grid(items * lpi);
-#define BA_DELTA_LAUNCH(T, L)                                                                              \
-    delta_kernel<T, L><<<grid, kThreads, 0, st>>>(items, op, gp, lse, delta_t, nlse2_t, row_begin, h_q,   \
-                                                  row_pitch)
+#define BA_DELTA_LAUNCH(T, L)                                                                            \
+    delta_kernel<T, L><<<grid, kThreads, 0, st>>>(items, items_a, op, gp, lse, delta_t, nlse2_t,        \
+                                                  row_a_begin, row_b_begin, h_q, row_pitch)
     if (dtype == BA_FP32 && lpi == 16) BA_DELTA_LAUNCH(float, 16);
     else if (dtype == BA_FP32 && lpi == 32) BA_DELTA_LAUNCH(float, 32);
     else if (dtype == BA_BF16 && lpi == 8) BA_DELTA_LAUNCH(__nv_bfloat16, 8);

@@ -57,8 +57,12 @@ struct PlanArgs {
     unsigned long long *pairs;
 };
 
+// Token offset of branch b.  With no branches (A = 0) there is no offsets array
+// to read -- the caller may have passed NULL -- and every offset is 0.
 __device__ __forceinline__ int32_t branch_offset(const PlanArgs &p, int32_t b) {
-    return p.uniform_len > 0 ? b * p.uniform_len : p.offs[b];
+    if (p.uniform_len > 0) return b * p.uniform_len;
+    if (p.a == 0 || p.offs == nullptr) return 0;
+    return p.offs[b];
 }
 
 // Largest s in [0, B) with cu[s] <= i and cu[s+1] > i (the non-empty sequence
@@ -234,7 +238,11 @@ extern "C" int ba_plan_create(const ba_problem_t *p, void *plan_mem, size_t plan
     PlanArgs a;
     a.n = p->n_main; a.m = p->n_branch; a.b = p->num_seqs; a.a = p->num_branches;
     a.kind = p->mask_kind; a.uniform_len = p->uniform_len;
-    a.cu = p->cu_seqlens; a.anchor = p->anchor_idx; a.offs = p->branch_offsets; a.parent = p->parent;
+    a.cu = p->cu_seqlens;
+    // A = 0: the branch arrays are never read, whatever the caller passed for them
+    a.anchor = p->num_branches > 0 ? p->anchor_idx : nullptr;
+    a.offs = (p->num_branches > 0 && p->uniform_len == 0) ? p->branch_offsets : nullptr;
+    a.parent = (p->mask_kind == BA_MASK_TREE && p->n_branch > 0) ? p->parent : nullptr;
     a.row_lo = (int32_t *)(base + l.row_lo); a.row_hi = (int32_t *)(base + l.row_hi);
     a.br_start = (int32_t *)(base + l.br_start); a.br_end = (int32_t *)(base + l.br_end);
     a.br_mask = (uint64_t *)(base + l.br_mask);

@@ -589,6 +589,13 @@ int ba_tc_bwd_fused(const ba_plan *pl, const BaRange &r, const void *q_main, con
     if (dev < 0 || dev >= 64) return BA_EUNSUPPORTED;
     const size_t smem = sizeof(FusedSmem);
     if (!attr_set[dev]) {
+        // The register re-split inside the kernel hands out what a launch with 128 registers per
+        // thread owns.  A build that gave the kernel fewer (another compiler, a register cap, a debug
+        // build) would leave setmaxnreg.inc waiting for registers nobody releases: refuse to launch.
+        cudaFuncAttributes fa;
+        BA_CUDA_CHECK(cudaFuncGetAttributes(&fa, tc_bwd_fused_kernel));
+        if (fa.numRegs * kFusedThreads < 2 * 128 * kRegsCompute + 128 * kRegsReduce + 128 * kRegsIssue)
+            return BA_EUNSUPPORTED;
         BA_CUDA_CHECK(cudaFuncSetAttribute(tc_bwd_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_set[dev] = true;
     }

@@ -92,11 +92,41 @@ def pairs_per_rank(problem, cp: int) -> List[int]:
     return out
 
 
-def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None):
+class Workspace:
+    """Device buffers of the emulated layout, allocated once and reused by every
+    step: the two compact fp32 (O, LSE) accumulators of a query chunk, and for the
+    backward the four fp32 gradient accumulators plus the gradients in the input
+    dtype.  (A step zeroes the accumulators with one memset each.)"""
+
+    def __init__(self, ba, plan, cp, backward=True):
+        import torch
+        p = plan.problem
+        self.cp = cp
+        dev = plan.device
+        csize = p.n_main // (2 * cp)
+        max_rows = 0
+        for b in schedule(p, cp):
+            t0, t1 = plan.token_range(*b.br)
+            max_rows = max(max_rows, csize + t1 - t0)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.acc_o = torch.empty((max_rows, p.h_q, p.head_dim), **f32)
+        self.acc_l = torch.empty((max_rows, p.h_q), **f32)
+        self.inc_o = self.inc_l = None
+        if plan.impl != ba.IMPL_TC:       # the plain-FMA path merges in a pass of its own
+            self.inc_o, self.inc_l = torch.empty_like(self.acc_o), torch.empty_like(self.acc_l)
+        self.grads = self.outs = None
+        if backward:
+            shapes = ((p.n_main, p.h_q, p.head_dim), (p.n_branch, p.h_q, p.head_dim),
+                      (p.rows, p.h_kv, p.head_dim), (p.rows, p.h_kv, p.head_dim))
+            self.grads = tuple(torch.empty(s, **f32) for s in shapes)
+            self.outs = tuple(torch.empty(s, dtype=plan.torch_dtype, device=dev) for s in shapes)
+
+
+def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None, ws=None):
     """Emulated CP forward: per (rank, step) partial calls, each merged into the
     running (O, LSE) by Eq. (lse-merge) -- in the kernel's epilogue on tensor-core
-    plans, by `lse_merge` otherwise.
-    Returns (O [N+M,h_q,D] input dtype, LSE fp32, number of library launches)."""
+    plans, by `lse_merge` otherwise.  `out` may be fp32 (no rounding of O).
+    Returns (O [N+M,h_q,D], LSE fp32, number of library launches)."""
     import torch
     p = plan.problem
     n = p.n_main
@@ -104,21 +134,16 @@ def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None):
         out = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=plan.device)
     if lse is None:
         lse = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=plan.device)
+    if ws is None:
+        ws = Workspace(ba, plan, cp, backward=False)
     blocks = schedule(p, cp)
     launches = 0
     # two compact fp32 buffers (accumulated, incoming) reused by every q chunk
     csize = n // (2 * cp)
-    max_rows = 0
-    for b in blocks:
-        t0, t1 = plan.token_range(*b.br)
-        max_rows = max(max_rows, csize + t1 - t0)
-    acc_o = torch.empty((max_rows, p.h_q, p.head_dim), dtype=torch.float32, device=plan.device)
-    acc_l = torch.empty((max_rows, p.h_q), dtype=torch.float32, device=plan.device)
+    acc_o, acc_l, inc_o, inc_l = ws.acc_o, ws.acc_l, ws.inc_o, ws.inc_l
     # tensor-core plans merge each later ring step into the accumulators in the kernel's
     # epilogue; the plain-FMA path writes the step's partial result and merges it in a pass of its own
     in_kernel = plan.impl == ba.IMPL_TC
-    inc_o = None if in_kernel else torch.empty_like(acc_o)
-    inc_l = None if in_kernel else torch.empty_like(acc_l)
     for rank in range(cp):
         for qc in rank_chunks(rank, cp):
             mine = [b for b in blocks if b.rank == rank and b.q_chunk == qc]
@@ -151,24 +176,37 @@ def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None):
     return out, lse, launches
 
 
-def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp, fused=False):
+def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp, fused=False, ws=None):
     """Emulated CP backward: the same (rank, step) blocks, gradients accumulated
     in fp32 and converted once at the end.  Returns (dQ_main, dQ_branch, dK, dV,
     launches) in the input dtype.  `fused`: one kernel per block for dQ, dK and
-    dV (dQ summed with atomic adds) instead of a dQ and a dK/dV kernel."""
-    import torch
+    dV (dQ summed with atomic adds) instead of a dQ and a dK/dV kernel.
+    The per-row scalars (delta and -LSE log2 e) of a query chunk are prepared once,
+    before the chunk's first block, not once per block."""
     p = plan.problem
-    f32 = dict(dtype=torch.float32, device=plan.device)
-    grads = (torch.zeros((p.n_main, p.h_q, p.head_dim), **f32),
-             torch.zeros((p.n_branch, p.h_q, p.head_dim), **f32),
-             torch.zeros((p.rows, p.h_kv, p.head_dim), **f32),
-             torch.zeros((p.rows, p.h_kv, p.head_dim), **f32))
+    if ws is None or ws.grads is None:
+        ws = Workspace(ba, plan, cp, backward=True)
+    grads = ws.grads
+    for g in grads:
+        g.zero_()
     launches = 0
-    for b in schedule(p, cp):
-        parts = ba.PART_MAIN | (ba.PART_BRANCH if b.branch_part else 0)
-        ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=b.qm, br_range=b.br,
-                           kv_range=b.kv, parts=parts, accumulate=True, grads=grads,
-                           stages=ba.STAGE_ALL_FUSED if fused else ba.STAGE_ALL)
-        launches += 3 if fused else 4
-    outs = tuple(ba.ba_finalize_grads(g, dtype=plan.torch_dtype) for g in grads)
+    common = dict(accumulate=True, grads=grads)
+    blocks = schedule(p, cp)
+    for rank in range(cp):
+        for qc in rank_chunks(rank, cp):
+            mine = [b for b in blocks if b.rank == rank and b.q_chunk == qc]
+            ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, qm_range=mine[0].qm, br_range=mine[0].br,
+                               kv_range=(0, 0), parts=0, stages=ba.STAGE_PREP, **common)
+            launches += 1
+            for b in mine:
+                parts = ba.PART_MAIN | (ba.PART_BRANCH if b.branch_part else 0)
+                rng = dict(qm_range=b.qm, br_range=b.br, kv_range=b.kv, parts=parts)
+                if fused:
+                    ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, stages=ba.STAGE_FUSED, **rng, **common)
+                    launches += 1
+                else:
+                    ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, stages=ba.STAGE_DQ, **rng, **common)
+                    ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, stages=ba.STAGE_DKDV, **rng, **common)
+                    launches += 2
+    outs = tuple(ba.ba_finalize_grads(g, dst=d) for g, d in zip(grads, ws.outs))
     return (*outs, launches + 4)

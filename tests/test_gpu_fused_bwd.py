@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2609_07108_b200 import workloads as W
-from helpers import TOL, assert_close, f32, oracle_fwd_bwd, to_dev
+from helpers import TOL, assert_close, f32, key_viewer_counts, oracle_fwd_bwd, to_dev, visible_counts
 
 pytestmark = pytest.mark.gpu
 
@@ -24,7 +24,7 @@ def fused_grads(ba, plan, d, o, lse, q_main=True, grads=None, **ranges):
                               grads=grads, stages=ba.STAGE_ALL_FUSED, **ranges)
 
 
-def check_fused(ba, oracle, p, seed=0, std=0.5, groups=None, q_main=True, mutate=None):
+def check_fused(ba, oracle, p, seed=0, std=0.5, groups=None, q_main=True, mutate=None, relative_grads=True):
     t = W.make_tensors(p, seed=seed, std=std)
     if mutate:
         mutate(t)
@@ -39,17 +39,19 @@ def check_fused(ba, oracle, p, seed=0, std=0.5, groups=None, q_main=True, mutate
     dqm, dqb, dk, dv = fused_grads(ba, plan, d, o, lse, q_main=q_main)
     plan.check()
     tol = TOL["bf16"]
+    nk, kk = visible_counts(p), key_viewer_counts(p)
+    rel = relative_grads
     if q_main:
-        assert_close("dQ_main", f32(dqm)[:, qh], ref["dq"][:n], tol)
-    assert_close("dQ_branch", f32(dqb)[:, qh], ref["dq"][n:], tol)
-    assert_close("dK", f32(dk)[:, kvh], ref["dk"], tol)
-    assert_close("dV", f32(dv)[:, kvh], ref["dv"], tol)
+        assert_close("dQ_main", f32(dqm)[:, qh], ref["dq"][:n], tol, row_keys=nk[:n], relative=rel)
+    assert_close("dQ_branch", f32(dqb)[:, qh], ref["dq"][n:], tol, row_keys=nk[n:], relative=rel)
+    assert_close("dK", f32(dk)[:, kvh], ref["dk"], tol, row_keys=kk, relative=rel)
+    assert_close("dV", f32(dv)[:, kvh], ref["dv"], tol, row_keys=kk)
     # the split kernels on the same inputs: same sums up to the order of the dQ terms
     split = ba.branch_attn_bwd(plan, d["q_main"] if q_main else None, d["q_branch"], d["k"], d["v"], o, lse,
                                d["d_o"], accumulate=True)
     for name, a, b in zip(("dQm", "dQb", "dK", "dV"), (dqm, dqb, dk, dv), split):
         if a is not None:
-            assert_close(name + " fused vs split", f32(a), f32(b).astype(np.float64), 5e-3)
+            assert_close(name + " fused vs split", f32(a), f32(b).astype(np.float64), 5e-3, relative=False)
     plan.check()
     # gradients in the input dtype: dQ summed in the workspace and converted, dK / dV stored directly
     gq, gb, gk, gv = ba.branch_attn_bwd(plan, d["q_main"] if q_main else None, d["q_branch"], d["k"], d["v"], o, lse,
@@ -57,10 +59,10 @@ def check_fused(ba, oracle, p, seed=0, std=0.5, groups=None, q_main=True, mutate
     plan.check()
     assert gb.dtype == torch.bfloat16 and gk.dtype == torch.bfloat16
     if q_main:
-        assert_close("dQ_main bf16", f32(gq)[:, qh], ref["dq"][:n], tol)
-    assert_close("dQ_branch bf16", f32(gb)[:, qh], ref["dq"][n:], tol)
-    assert_close("dK bf16", f32(gk)[:, kvh], ref["dk"], tol)
-    assert_close("dV bf16", f32(gv)[:, kvh], ref["dv"], tol)
+        assert_close("dQ_main bf16", f32(gq)[:, qh], ref["dq"][:n], tol, row_keys=nk[:n], relative=rel)
+    assert_close("dQ_branch bf16", f32(gb)[:, qh], ref["dq"][n:], tol, row_keys=nk[n:], relative=rel)
+    assert_close("dK bf16", f32(gk)[:, kvh], ref["dk"], tol, row_keys=kk, relative=rel)
+    assert_close("dV bf16", f32(gv)[:, kvh], ref["dv"], tol, row_keys=kk)
 
 
 @pytest.mark.parametrize("kind", [W.CHAIN, W.BLOCK, W.TREE])
@@ -103,7 +105,7 @@ def _late_outlier(t):   # one key aligned with a late query
 @pytest.mark.parametrize("mutate", [_sharp, _offset, _late_outlier])
 def test_stress_inputs(ba, oracle, mutate):
     p = W.odd_shapes(W.CHAIN, head_dim=128, dtype="bf16", h_q=4, h_kv=2)
-    check_fused(ba, oracle, p, seed=6, mutate=mutate)
+    check_fused(ba, oracle, p, seed=6, mutate=mutate, relative_grads=mutate is _offset)
 
 
 def test_unaligned_ranges_with_gradients_in_the_input_dtype(ba, oracle):
@@ -126,12 +128,13 @@ def test_unaligned_ranges_with_gradients_in_the_input_dtype(ba, oracle):
                        kv_range=kv, grads=grads, stages=ba.STAGE_ALL_FUSED)
     plan.check()
     dq = torch.cat([grads[0], grads[1]], 0)
-    assert_close("dQ (selected rows)", f32(dq)[rows], ref_dq, TOL["bf16"])
+    nk, kk = visible_counts(p), key_viewer_counts(p)
+    assert_close("dQ (selected rows)", f32(dq)[rows], ref_dq, TOL["bf16"], row_keys=nk[rows])
     other = np.ones(p.rows, bool); other[rows] = False
     assert float((dq[torch.from_numpy(other).cuda()].float() - 7.0).abs().max()) == 0.0
     keys = np.concatenate([np.arange(*kv), n + np.arange(t0, t1)])       # the key set of the call
-    assert_close("dK (key set)", f32(grads[2])[keys], ref_dk[keys], TOL["bf16"])
-    assert_close("dV (key set)", f32(grads[3])[keys], ref_dv[keys], TOL["bf16"])
+    assert_close("dK (key set)", f32(grads[2])[keys], ref_dk[keys], TOL["bf16"], row_keys=kk[keys])
+    assert_close("dV (key set)", f32(grads[3])[keys], ref_dv[keys], TOL["bf16"], row_keys=kk[keys])
 
 
 def test_no_branches(ba, oracle):
@@ -157,9 +160,10 @@ def test_key_chunks_and_query_ranges_accumulate(ba, oracle):
     plan.check()
     ref = oracle_fwd_bwd(oracle, p, t)
     want = (ref["dq"][:n], ref["dq"][n:], ref["dk"], ref["dv"])
-    for name, g, w in zip(("dQm", "dQb", "dK", "dV"), grads, want):
-        assert_close(name, f32(g), w, TOL["bf16"])
-        assert_close(name + " finalized", f32(ba.ba_finalize_grads(g, dtype=torch.bfloat16)), w, TOL["bf16"])
+    nk, kk = visible_counts(p), key_viewer_counts(p)
+    for name, g, w, rk in zip(("dQm", "dQb", "dK", "dV"), grads, want, (nk[:n], nk[n:], kk, kk)):
+        assert_close(name, f32(g), w, TOL["bf16"], row_keys=rk)
+        assert_close(name + " finalized", f32(ba.ba_finalize_grads(g, dtype=torch.bfloat16)), w, TOL["bf16"], row_keys=rk)
 
 
 def test_dk_dv_bit_identical_dq_close_run_to_run(ba):

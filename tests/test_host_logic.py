@@ -118,3 +118,34 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.lse_merge(-1, 128, None, None, None, None, None, 1, None, None) == -1
     assert lib.ba_finalize_grads(None, None, 0, 0, None) == 0
     assert lib.branch_attn_fwd(None, None, None, None, None, None, None, None, 0, None) == -1
+
+
+def test_closed_form_helpers_agree_with_brute_force():
+    from helpers import GROUP_OFFSET, N_BITS, branch_visibility, expected_bit_fractions, visible_counts
+    """The closed forms themselves, on a small tree batch, against explicit enumeration."""
+    p = W.config4(shrink=64)
+    vis_b = branch_visibility(p)
+    cu = p.cu_seqlens.astype(np.int64)
+    n = p.n_main
+    for g in (0, 3):
+        exp = expected_bit_fractions(p, g)
+        rng = np.random.default_rng(0)
+        for r in rng.choice(p.rows, size=40, replace=False):
+            if r < n:
+                s = np.searchsorted(cu, r, side="right") - 1
+                keys = list(range(cu[s], r + 1))
+            else:
+                tkn = r - n
+                b = tkn // 31
+                a = int(p.anchor_idx[b])
+                s = np.searchsorted(cu, a, side="right") - 1
+                keys = list(range(cu[s], a + 1))
+                node = tkn - 31 * b
+                while node >= 0:
+                    keys.append(n + 31 * b + node)
+                    node = int(p.parent[31 * b + node])
+                assert sorted(k - n - 31 * b for k in keys if k >= n) == list(np.nonzero(vis_b[tkn])[0])
+            codes = np.array(keys, dtype=np.int64) + g * GROUP_OFFSET
+            assert len(keys) == visible_counts(p)[r]
+            for c in range(N_BITS):
+                assert abs(((codes >> c) & 1).mean() - exp[r, c]) < 1e-12

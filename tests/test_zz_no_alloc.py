@@ -52,8 +52,13 @@ def test_static_scratch_backward_rejects_problems_beyond_its_limit():
     p = W.config3()                              # 40,960 rows x 32 heads: 10.5 MB of scratch > 8 MiB
     plan = ba.Plan(p)
     assert ba._lib().ba_workspace_bytes(plan.handle, ba.OP_BWD) > ba.STATIC_SCRATCH_BYTES
-    dummy = torch.zeros(16, device="cuda")
-    with pytest.raises(ba.BranchAttnError) as e:
-        ba.branch_attn_bwd_static(plan, dummy, dummy, dummy, dummy, dummy, dummy, dummy,
-                                  grads=(dummy, dummy, dummy, dummy))
+    def empty(*shape, dtype=torch.bfloat16):
+        return torch.empty(shape, dtype=dtype, device="cuda")
+
+    n, m, r = p.n_main, p.n_branch, p.rows
+    hq, hkv, d = p.h_q, p.h_kv, p.head_dim
+    with pytest.raises(ba.BranchAttnError) as e:       # refused before anything is launched
+        ba.branch_attn_bwd_static(plan, empty(n, hq, d), empty(m, hq, d), empty(r, hkv, d), empty(r, hkv, d),
+                                  empty(r, hq, d), empty(r, hq, dtype=torch.float32), empty(r, hq, d),
+                                  grads=(empty(n, hq, d), empty(m, hq, d), empty(r, hkv, d), empty(r, hkv, d)))
     assert e.value.code == -3
