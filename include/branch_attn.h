@@ -122,6 +122,17 @@ int ba_plan_impl(const ba_plan_t *plan);
 int ba_plan_check(ba_plan_t *plan, void *stream);
 
 /*
+ * Self-test of the bounded device-side waits (no counterpart in the paper: every
+ * barrier wait inside the tensor-core kernels gives up after a cycle limit instead of
+ * spinning forever, and this shows that path working).  Launches one warp that
+ * waits, for at most `limit_cycles` SM cycles (1 .. 1e8, i.e. well under a tenth of
+ * a second), on a barrier nobody signals; the kernel then returns normally and
+ * leaves BA_ETIMEOUT in the plan's status word, which the next ba_plan_check
+ * reports and clears.  Nothing else is touched; later calls work as usual.
+ */
+int ba_selftest_bounded_wait(ba_plan_t *plan, int64_t limit_cycles, void *stream);
+
+/*
  * Forward, both key sets fused in one online-softmax pass (Section 3.2: the
  * causal main-sequence component and the branch-local component; Eq.
  * (lse-merge) applied tile by tile).

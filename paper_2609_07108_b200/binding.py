@@ -48,7 +48,7 @@ _LIB = None
 EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
            "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "ba_plan_check", "branch_attn_fwd",
            "branch_attn_fwd_partial", "branch_attn_fwd_partial_merge", "lse_merge", "branch_attn_bwd", "branch_attn_bwd_stages",
-           "branch_attn_bwd_static", "ba_finalize_grads")
+           "branch_attn_bwd_static", "ba_finalize_grads", "ba_selftest_bounded_wait")
 
 
 def _lib():
@@ -97,6 +97,8 @@ def _lib():
         lib.branch_attn_bwd_static.argtypes = lib.branch_attn_bwd.argtypes[:-3] + [vp]
         lib.ba_finalize_grads.restype = C.c_int
         lib.ba_finalize_grads.argtypes = [vp, vp, i64, C.c_int, vp]
+        lib.ba_selftest_bounded_wait.restype = C.c_int
+        lib.ba_selftest_bounded_wait.argtypes = [vp, i64, vp]
         _LIB = lib
     return _LIB
 
@@ -194,6 +196,10 @@ class Plan:
     def check(self):
         """Synchronise and raise if a kernel of this plan gave up a bounded wait."""
         _check(_lib().ba_plan_check(self.handle, _stream()), "ba_plan_check")
+
+    def selftest_bounded_wait(self, limit_cycles=100000):
+        """Launch the probe whose wait runs out; the next `check()` raises BA_ETIMEOUT."""
+        _check(_lib().ba_selftest_bounded_wait(self.handle, limit_cycles, _stream()), "ba_selftest_bounded_wait")
 
     def close(self):
         if getattr(self, "handle", None):

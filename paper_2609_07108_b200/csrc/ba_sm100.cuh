@@ -57,7 +57,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // wait would sit on the critical path of each producer/consumer handoff); the
 // limit is in SM cycles, about two seconds.
 constexpr long long kWaitLimitCycles = 4000000000ll;
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles) {
     long long t0 = 0;
 #pragma unroll 1
     for (uint32_t spins = 1;; ++spins) {
@@ -66,7 +67,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitCycles) {
+            if (now - t0 > limit_cycles) {
                 *abort_flag = 1;
                 return false;
             }

@@ -136,20 +136,24 @@ def visible_counts(p):
 
 
 def key_viewer_counts(p):
-    """For every key (main keys, then branch tokens): the largest visible-set size
-    among the query rows that can see it -- the length of its sequence for a main
-    key, prefix + branch length for a branch key.  Keys whose every viewer has
-    only a few keys inherit the cancellation described at ROW_GATE_MIN_KEYS."""
+    """For every key (main keys, then branch tokens): an upper bound on the largest
+    visible-set size among the query rows that can see it -- the longest row of its
+    sequence for a main key, the longest row of its own branch for a branch key.  Keys
+    whose every viewer has only a few keys inherit the cancellation described at
+    ROW_GATE_MIN_KEYS."""
     cu = p.cu_seqlens.astype(np.int64)
     pos = np.arange(p.n_main, dtype=np.int64)
     seq = np.searchsorted(cu, pos, side="right") - 1
     main = cu[seq + 1] - cu[seq]
     if p.num_branches == 0:
         return main
-    anchors = p.anchor_idx.astype(np.int64)
-    aseq = np.searchsorted(cu, anchors, side="right") - 1
-    blen = np.diff(p.branch_offsets.astype(np.int64))
-    return np.concatenate([main, np.repeat(anchors - cu[aseq] + 1 + blen, blen)])
+    nk = visible_counts(p)[p.n_main:]
+    offs = p.branch_offsets.astype(np.int64)
+    blen = np.diff(offs)
+    longest = np.zeros(p.num_branches, dtype=np.int64)
+    nonempty = blen > 0
+    longest[nonempty] = np.maximum.reduceat(nk, offs[:-1][nonempty])
+    return np.concatenate([main, np.repeat(longest, blen)])
 
 
 # Closed forms of the visible sets (q = 0 probes of the full-size tests), from the metadata alone.

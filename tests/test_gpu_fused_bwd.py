@@ -105,7 +105,7 @@ def _late_outlier(t):   # one key aligned with a late query
 @pytest.mark.parametrize("mutate", [_sharp, _offset, _late_outlier])
 def test_stress_inputs(ba, oracle, mutate):
     p = W.odd_shapes(W.CHAIN, head_dim=128, dtype="bf16", h_q=4, h_kv=2)
-    check_fused(ba, oracle, p, seed=6, mutate=mutate, relative_grads=mutate is _offset)
+    check_fused(ba, oracle, p, seed=6, mutate=mutate, relative_grads=False)
 
 
 def test_unaligned_ranges_with_gradients_in_the_input_dtype(ba, oracle):
