@@ -44,6 +44,10 @@ WORKLOADS = {
     "config2_eagle3_8k": (2, 1, 0, False),
     # shape of the paper's packed variable-length operator benchmark (longest sequence 20,480 tokens)
     "varlen_ttt_72k": (6, 1, 0, True),
+    # the same shape through the step-major calls: main rows, then depth 1, 2, 3 in turn
+    "varlen_ttt_72k_stepwise": (6, 1, "stepwise", True),
+    # config 5 through the K/V ring driver (shards copied into a local double buffer on a side stream)
+    "config5_256k_ring": (5, 1, ("ring", 8), True),
 }
 
 
@@ -261,6 +265,20 @@ class Recorder:
     def ba_finalize_grads(self, *a, **k):
         return self._wrap("finalize", 1, self.ba.ba_finalize_grads, *a, **k)
 
+    def branch_attn_fwd_shard(self, *a, **k):
+        return self._wrap("fwd", 1, self.ba.branch_attn_fwd_shard, *a, **k)
+
+    def branch_attn_bwd_shard(self, *a, **k):
+        ba = self.ba
+        kind = {ba.STAGE_DQ: "bwd_dq", ba.STAGE_DKDV: "bwd_dkdv", ba.STAGE_FUSED: "bwd_fused"}[k["stages"]]
+        return self._wrap(kind, 1, ba.branch_attn_bwd_shard, *a, **k)
+
+    def branch_attn_fwd_depth(self, *a, **k):
+        return self._wrap("fwd", 1, self.ba.branch_attn_fwd_depth, *a, **k)
+
+    def branch_attn_bwd_depth(self, *a, **k):     # delta, the one-kernel backward, conversion of dQ
+        return self._wrap("bwd_depth", 3, self.ba.branch_attn_bwd_depth, *a, **k)
+
     def totals(self):
         out = {}
         for kind, s, e in self.events:
@@ -286,7 +304,14 @@ def make_device_inputs(p, torch, device, seed=0):
 
 
 def run_fwd(rec, plan, t, cp):
-    from paper_2609_07108_b200 import zigzag
+    from paper_2609_07108_b200 import ring, zigzag
+    mode = t.get("_mode", "zigzag" if cp else "mono")
+    if mode == "stepwise":
+        return stepwise_fwd(rec, plan, t)
+    if mode == "ring":
+        o, lse, _ = ring.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp, out=t.get("_o"),
+                                 lse=t.get("_lse"), ws=t.get("_ws"), bufs=t["_bufs"], stats=t.get("_ring_stats"))
+        return o, lse
     if cp:
         o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp,
                                    out=t.get("_o"), lse=t.get("_lse"), ws=t.get("_ws"))
@@ -295,7 +320,13 @@ def run_fwd(rec, plan, t, cp):
 
 
 def run_bwd(rec, plan, t, cp, o, lse, fused=False):
-    from paper_2609_07108_b200 import zigzag
+    from paper_2609_07108_b200 import ring, zigzag
+    mode = t.get("_mode", "zigzag" if cp else "mono")
+    if mode == "stepwise":
+        return stepwise_bwd(rec, plan, t, o, lse, fused)
+    if mode == "ring":
+        return ring.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp,
+                             fused=fused, ws=t.get("_ws"), bufs=t["_bufs"], stats=t.get("_ring_stats"))
     if cp:
         return zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp,
                                fused=fused, ws=t.get("_ws"))
@@ -307,6 +338,66 @@ def run_step(rec, plan, t, cp, backward, fused=False):
     o, lse = run_fwd(rec, plan, t, cp)
     grads = run_bwd(rec, plan, t, cp, o, lse, fused=fused) if backward else None
     return o, lse, grads
+
+
+# ---- the step-major form: the main rows through a branch-free plan, then one call per depth
+# (a trainer produces the depth-d tokens only after depth d - 1), branch K / V stored depth-major
+
+def stepwise_setup(ba, plan, p, t, torch, device):
+    n, a, length = p.n_main, p.num_branches, int(p.branch_offsets[1])
+    main_p = W.Problem(p.cu_seqlens, np.zeros(0, np.int32), np.zeros(1, np.int32), W.CHAIN, None, p.h_q, p.h_kv,
+                       p.head_dim, dtype=p.dtype, name=p.name + "_main_rows")
+    s = {"plan_main": ba.Plan(main_p, device=device, impl=plan.impl), "n": n, "a": a, "len": length}
+    hq, hkv, d = p.h_q, p.h_kv, p.head_dim
+    dt = plan.torch_dtype
+    # the same random values, regrouped: queries / cotangents per depth, branch keys depth-major
+    s["q_d"] = [t["q_branch"].reshape(a, length, hq, d)[:, j].contiguous() for j in range(length)]
+    s["go_main"] = t["d_o"][:n].contiguous()
+    s["go_d"] = [t["d_o"][n:].reshape(a, length, hq, d)[:, j].contiguous() for j in range(length)]
+
+    def dm(x):
+        return torch.cat([x[:n], x[n:].reshape(a, length, hkv, d).transpose(0, 1).reshape(a * length, hkv, d)], 0).contiguous()
+
+    s["k"], s["v"] = dm(t["k"]), dm(t["v"])
+    s["k_main"], s["v_main"] = s["k"][:n], s["v"][:n]
+    s["o_main"] = torch.empty((n, hq, d), dtype=dt, device=device)
+    s["lse_main"] = torch.empty((n, hq), dtype=torch.float32, device=device)
+    s["o_d"] = [torch.empty((a, hq, d), dtype=dt, device=device) for _ in range(length)]
+    s["lse_d"] = [torch.empty((a, hq), dtype=torch.float32, device=device) for _ in range(length)]
+    s["dq_main32"] = torch.empty((n, hq, d), dtype=torch.float32, device=device)
+    s["dq_main"] = torch.empty((n, hq, d), dtype=dt, device=device)
+    s["dq_d"] = [torch.empty((a, hq, d), dtype=dt, device=device) for _ in range(length)]
+    s["dk32"] = torch.empty((p.rows, hkv, d), dtype=torch.float32, device=device)
+    s["dv32"] = torch.empty((p.rows, hkv, d), dtype=torch.float32, device=device)
+    s["dk"] = torch.empty((p.rows, hkv, d), dtype=dt, device=device)
+    s["dv"] = torch.empty((p.rows, hkv, d), dtype=dt, device=device)
+    s["none"] = torch.empty((0, hq, d), dtype=torch.float32, device=device)
+    return s
+
+
+def stepwise_fwd(rec, plan, t):
+    s = t["_sw"]
+    rec.branch_attn_fwd(s["plan_main"], t["q_main"], None, s["k_main"], s["v_main"], out=s["o_main"], lse=s["lse_main"])
+    for j in range(s["len"]):
+        rec.branch_attn_fwd_depth(plan, j + 1, s["q_d"][j], s["k"], s["v"], out=s["o_d"][j], lse=s["lse_d"][j])
+    return s["o_main"], s["lse_main"]
+
+
+def stepwise_bwd(rec, plan, t, o, lse, fused):
+    s = t["_sw"]
+    n = s["n"]
+    for x in (s["dq_main32"], s["dk32"], s["dv32"]):
+        x.zero_()
+    for j in reversed(range(s["len"])):            # deepest first, as backpropagation reaches them
+        rec.branch_attn_bwd_depth(plan, j + 1, s["q_d"][j], s["k"], s["v"], s["o_d"][j], s["lse_d"][j], s["go_d"][j],
+                                  s["dk32"], s["dv32"], dq=s["dq_d"][j])
+    rec.branch_attn_bwd(s["plan_main"], t["q_main"], None, s["k_main"], s["v_main"], o, lse, s["go_main"],
+                        accumulate=True, grads=(s["dq_main32"], s["none"], s["dk32"][:n], s["dv32"][:n]),
+                        stages=rec.STAGE_ALL_FUSED if fused else rec.STAGE_ALL)
+    rec.ba_finalize_grads(s["dq_main32"], dst=s["dq_main"])
+    rec.ba_finalize_grads(s["dk32"], dst=s["dk"])
+    rec.ba_finalize_grads(s["dv32"], dst=s["dv"])
+    return s["dq_main"], s["dq_d"], s["dk"], s["dv"]
 
 
 def use_fused_bwd(args, p, plan, ba):
@@ -328,6 +419,11 @@ def run_ours(args):
     if name == "auto":
         name = "config5_256k_zigzag"
     cfg, shrink, cp, backward = WORKLOADS[name]
+    mode = "zigzag" if cp else "mono"
+    if cp == "stepwise":
+        mode, cp = "stepwise", 0
+    elif isinstance(cp, tuple):
+        mode, cp = cp
     p = W.CONFIGS[cfg](shrink) if cfg != 1 else W.config1()
     impl = {"auto": ba.IMPL_AUTO, "simt": ba.IMPL_SIMT, "tc": ba.IMPL_TC}[args.kernels]
     plan = ba.Plan(p, device=device, impl=impl)
@@ -352,9 +448,14 @@ def run_ours(args):
     # outputs and (zigzag) the fp32 accumulators are allocated once, outside the steps
     t["_o"] = torch.empty((p.rows, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
     t["_lse"] = torch.empty((p.rows, p.h_q), dtype=torch.float32, device=device)
-    if cp:
-        from paper_2609_07108_b200 import zigzag
+    t["_mode"] = mode
+    if mode == "stepwise":
+        t["_sw"] = stepwise_setup(ba, plan, p, t, torch, device)
+    elif cp:
+        from paper_2609_07108_b200 import ring, zigzag
         t["_ws"] = zigzag.Workspace(ba, plan, cp, backward=backward)
+        if mode == "ring":
+            t["_bufs"] = ring.RingBuffers(plan, cp)
     elif backward:
         t["_grads"] = (torch.empty((p.n_main, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=device)
                        if not branch_only else None,
@@ -384,6 +485,9 @@ def run_ours(args):
         sampler.start()
     rec.enabled = True
     step_ms = []
+    if mode == "ring":
+        from paper_2609_07108_b200 import ring
+        t["_ring_stats"] = ring.new_stats()
     barrier()
     for _ in range(args.steps):
         if flush is not None:
@@ -401,17 +505,44 @@ def run_ours(args):
     value, total_ms = aggregate_throughput(dist, flops * args.steps, local_ms, device)
     totals = rec.totals()
     launches = rec.launches
+    ring_report = None
+    if mode == "ring":
+        # Eq. (cp-comm) volume, the copies' own device time, and the exposed part: this driver's step
+        # against the same kernels run without any copy (the range-based zigzag driver)
+        stats = t.pop("_ring_stats")
+        t["_mode"] = "zigzag"
+        s0 = torch.cuda.Event(enable_timing=True)
+        e0 = torch.cuda.Event(enable_timing=True)
+        s0.record()
+        run_step(Recorder(ba, p), plan, t, cp, backward, fused=fused)
+        e0.record()
+        torch.cuda.synchronize()
+        t["_mode"] = "ring"
+        zz_ms = s0.elapsed_time(e0)
+        ring_ms = local_ms / args.steps
+        passes = (2 if backward else 1) * args.steps          # the backward replays the ring
+        copy_total = ring.copy_ms(stats)
+        n_copies = len(stats["copies"])
+        ring_report = {
+            "shard_bytes_per_rank_per_pass": ring.shard_bytes_per_rank(p, cp, 2),
+            "copied_bytes_per_rank_per_pass": stats["copied_bytes"] // (cp * passes),
+            "t_comm_ms_per_ring_step": round(copy_total / max(n_copies, 1), 4),
+            "t_attn_ms_per_ring_step": round((ring_ms - 0.0) / ((2 if backward else 1) * cp * cp), 4),
+            "step_ms_ring": round(ring_ms, 3), "step_ms_without_copies": round(zz_ms, 3),
+            "exposed_ms_per_step": round(ring_ms - zz_ms, 3),
+            "model": "Eq. cp-overlap: ring step time = max(t_comm, t_attn); exposed = max(0, t_comm - t_attn)",
+            "transport": "device copies into a local double buffer on one GPU; unmeasured over NVLink"}
 
     # ---- CPU baseline (the oracle on a bounded sample of the same inputs) and the GPU's error
     # against it on those rows; before the end-to-end run, which overwrites inputs and outputs
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(p, seconds_target=15.0, backward=backward,
-                           gpu=None if branch_only else (t, last))
+                           gpu=None if (branch_only or mode == "stepwise") else (t, last))
 
     # ---- end to end through the API with HOST buffers (pinned), copies timed
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and mode != "stepwise":
         e2e = run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args)
 
     # ---- dominant kernel and its roofline
@@ -424,11 +555,16 @@ def run_ours(args):
         # flop per visible pair and query head that the kernel itself executes, in
         # units of head_dim: forward 2 GEMMs (QK^T, PV); dQ kernel 3 (S, dP, dQ);
         # dK/dV kernel 4 (S^T and dP^T recomputed, dV, dK)
-        share = {"fwd": 4.0, "bwd_dq": 6.0, "bwd_dkdv": 8.0, "bwd_fused": 10.0}.get(kind)
+        share = {"fwd": 4.0, "bwd_dq": 6.0, "bwd_dkdv": 8.0, "bwd_fused": 10.0, "bwd_depth": 10.0}.get(kind)
         kernel_name = {"fwd": "tc_fwd_kernel", "bwd_dq": "tc_dq_kernel", "bwd_dkdv": "tc_dkdv_kernel",
-                       "bwd_fused": "tc_bwd_fused_kernel"}.get(kind, kind)
+                       "bwd_fused": "tc_bwd_fused_kernel", "bwd_depth": "tc_bwd_fused_kernel"}.get(kind, kind)
         if share is not None:
-            kflops = pairs * p.head_dim * p.h_q * share * args.steps
+            kpairs = pairs
+            if mode == "stepwise" and kind != "fwd":    # the per-depth calls cover the branch rows only
+                lens = np.diff(p.cu_seqlens.astype(np.int64))
+                main_pairs = int((lens * (lens + 1) // 2).sum())
+                kpairs = pairs - main_pairs if kind == "bwd_depth" else main_pairs
+            kflops = kpairs * p.head_dim * p.h_q * share * args.steps
             achieved = kflops / (ms * 1e-3) / 1e12
             long_step = total_ms / args.steps > 1000.0
             # query rows (row, head) one launch streams on average, for scaling the ncu traffic capture
@@ -462,7 +598,10 @@ def run_ours(args):
                        "path": (f"zigzag cp={cp}: partial fwd merged by Eq. lse-merge "
                                 + ("in the kernel epilogue" if plan.impl == ba.IMPL_TC else "with lse_merge")
                                 + ", partial bwd accumulate"
-                                if cp else "monolithic fwd + bwd"),
+                                + (", K/V shards of the remote ring steps copied into a local double buffer "
+                                   "on a side stream" if mode == "ring" else "")
+                                if cp else "step-major: main rows, then one call per depth (depth-major branch K/V)"
+                                if mode == "stepwise" else "monolithic fwd + bwd"),
                        "backward": backward,
                        "bwd_kernels": ("one fused kernel (dQ by fp32 atomic adds)" if fused
                                        else "dQ kernel + dK/dV kernel") if backward else None,
@@ -482,6 +621,8 @@ def run_ours(args):
             "roofline": roof,
             "cpu_baseline": cpu,
         }
+        if ring_report is not None:
+            line["ring"] = ring_report
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -49,7 +49,7 @@ typedef enum ba_status {
 enum { BA_BF16 = 0, BA_FP32 = 1 };
 enum { BA_MASK_CHAIN = 0, BA_MASK_BLOCK = 1, BA_MASK_TREE = 2 };
 enum { BA_PART_MAIN = 1, BA_PART_BRANCH = 2 };
-enum { BA_OP_FWD = 0, BA_OP_BWD = 1, BA_OP_BWD_FUSED = 2 };
+enum { BA_OP_FWD = 0, BA_OP_BWD = 1, BA_OP_BWD_FUSED = 2, BA_OP_BWD_DEPTH = 3 };
 enum { BA_STAGE_PREP = 1, BA_STAGE_DQ = 2, BA_STAGE_DKDV = 4, BA_STAGE_ALL = 7,
        BA_STAGE_FUSED = 8, BA_STAGE_ALL_FUSED = 9 };
 
@@ -106,7 +106,8 @@ int ba_plan_destroy(ba_plan_t *plan);
 /* Scratch bytes (device, 256-byte aligned) that `op` needs; may be 0.
  * BA_OP_BWD_FUSED = BA_OP_BWD plus an fp32 dQ accumulator of (N + M) * h_q * head_dim
  * floats: what BA_STAGE_FUSED needs when the gradients are written in the input
- * dtype (accumulate = 0). */
+ * dtype (accumulate = 0).  BA_OP_BWD_DEPTH = BA_OP_BWD plus an fp32 dQ accumulator of
+ * num_branches * h_q * head_dim floats (branch_attn_bwd_depth). */
 size_t ba_workspace_bytes(const ba_plan_t *plan, int op);
 
 /* Exact number of (query row, visible key) pairs per query head of the whole
@@ -272,6 +273,73 @@ int branch_attn_bwd_static(const ba_plan_t *plan, const void *q_main, const void
                            int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
                            int64_t kv_begin, int64_t kv_end, int parts, int accumulate,
                            void *dQ_main, void *dQ_branch, void *dK, void *dV, void *stream);
+
+/*
+ * One ring step on a RECEIVED K/V shard (Section 3.2, "Communication cost and
+ * overlap": K/V shards circulate between the context-parallel ranks while the
+ * queries stay local; Eq. (cp-comm) counts the shard bytes).  The same partial
+ * forward / backward as above for the causal-prefix keys only (BA_PART_MAIN), but
+ * the keys come from a buffer that holds just the shard:
+ *   k_shard, v_shard  [kv_end - kv_begin, h_kv, D]: main key rows [kv_begin,
+ *                     kv_end) as received (e.g. in a local double buffer); both
+ *                     ends must be multiples of 128 (kv_end may also be N),
+ *                     else BA_EINVAL.  Nothing outside the shard is read.
+ *   forward:  merge = 0 writes the compact fp32 partial (O_acc, LSE_acc) as
+ *             branch_attn_fwd_partial does, merge = 1 merges it into them as
+ *             branch_attn_fwd_partial_merge does.
+ *   backward: always accumulates.  dQ_main / dQ_branch are the local fp32
+ *             accumulators (global layout); dK_shard, dV_shard
+ *             [kv_end - kv_begin, h_kv, D] fp32 are the shard's gradient
+ *             accumulators, which travel around the ring with the shard and
+ *             return to its owner.  `stages` as in branch_attn_bwd_stages.
+ * The branch-local keys never move: the owner handles them in its local step
+ * with the calls above.
+ */
+int branch_attn_fwd_shard(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                          const void *k_shard, const void *v_shard,
+                          int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                          int64_t kv_begin, int64_t kv_end, int merge,
+                          float *O_acc, float *LSE_acc, void *stream);
+int branch_attn_bwd_shard(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                          const void *k_shard, const void *v_shard, const void *O, const float *LSE,
+                          const void *dO,
+                          int64_t qm_begin, int64_t qm_end, int64_t br_begin, int64_t br_end,
+                          int64_t kv_begin, int64_t kv_end,
+                          float *dQ_main, float *dQ_branch, float *dK_shard, float *dV_shard,
+                          void *workspace, size_t ws_bytes, void *stream, int stages);
+
+/*
+ * Step-major (per-depth) calls for training-time-test drafts (Section 3.2, draft
+ * families: the EAGLE-3 style draft feeds its own previous prediction back over
+ * several steps, so the tokens of depth d exist only after depth d - 1 has been
+ * computed; a trainer therefore needs one attention call per depth).
+ *
+ * Plan: BA_MASK_CHAIN with uniform_len = number of depths n, tensor-core kernels
+ * (bf16, head_dim 128); otherwise BA_EUNSUPPORTED.  `depth` is 1 .. n.
+ * Layout (depth-major, unlike the all-depths calls above):
+ *   q_depth, O_depth, dO_depth, dQ_depth  [A, h_q, D]   row b = the depth-`depth`
+ *                                         token of branch b;  LSE_depth [A, h_q]
+ *   k, v     [N + n * A, h_kv, D]  main rows, then the branch tokens of depth 1
+ *            (A rows, branch order), of depth 2, ...  Only the rows of depths
+ *            <= depth are read: later rows need not be written yet.
+ *   dK, dV   fp32, same layout as k, v; the terms of this call are ADDED (zero
+ *            them before the first call of a backward pass, convert with
+ *            ba_finalize_grads after the last).
+ * Query b sees the main keys of its causal prefix (up to and including its
+ * anchor) and the tokens of depths 1 .. depth of its own branch.  Branches
+ * [br_begin, br_end) are computed; other rows of the outputs are left alone.
+ * Running depth = 1 .. n over all branches gives the rows of branch_attn_fwd;
+ * the backward calls together (plus the main rows' own backward) give its
+ * gradients.  dQ_depth is summed with fp32 atomic adds and converted (as in
+ * BA_STAGE_FUSED).  workspace: ba_workspace_bytes(plan, BA_OP_BWD_DEPTH).
+ */
+int branch_attn_fwd_depth(const ba_plan_t *plan, int depth, const void *q_depth, const void *k,
+                          const void *v, int64_t br_begin, int64_t br_end, void *O_depth,
+                          float *LSE_depth, void *stream);
+int branch_attn_bwd_depth(const ba_plan_t *plan, int depth, const void *q_depth, const void *k,
+                          const void *v, const void *O_depth, const float *LSE_depth,
+                          const void *dO_depth, int64_t br_begin, int64_t br_end, void *dQ_depth,
+                          float *dK, float *dV, void *workspace, size_t ws_bytes, void *stream);
 
 /* fp32 accumulators -> dst_dtype (round to nearest even), `count` elements. */
 int ba_finalize_grads(const float *src, void *dst, int64_t count, int dst_dtype, void *stream);

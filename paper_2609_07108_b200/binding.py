@@ -17,7 +17,7 @@ from . import build as _build
 
 BA_BF16, BA_FP32 = 0, 1
 PART_MAIN, PART_BRANCH, PART_ALL = 1, 2, 3
-OP_FWD, OP_BWD, OP_BWD_FUSED = 0, 1, 2
+OP_FWD, OP_BWD, OP_BWD_FUSED, OP_BWD_DEPTH = 0, 1, 2, 3
 STAGE_PREP, STAGE_DQ, STAGE_DKDV, STAGE_ALL = 1, 2, 4, 7
 STAGE_FUSED, STAGE_ALL_FUSED = 8, 9
 IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
@@ -48,7 +48,8 @@ _LIB = None
 EXPORTS = ("ba_status_string", "ba_last_cuda_error", "ba_plan_bytes", "ba_plan_create",
            "ba_plan_destroy", "ba_workspace_bytes", "ba_plan_pairs", "ba_plan_impl", "ba_plan_check", "branch_attn_fwd",
            "branch_attn_fwd_partial", "branch_attn_fwd_partial_merge", "lse_merge", "branch_attn_bwd", "branch_attn_bwd_stages",
-           "branch_attn_bwd_static", "ba_finalize_grads", "ba_selftest_bounded_wait")
+           "branch_attn_bwd_static", "ba_finalize_grads", "ba_selftest_bounded_wait",
+           "branch_attn_fwd_depth", "branch_attn_bwd_depth", "branch_attn_fwd_shard", "branch_attn_bwd_shard")
 
 
 def _lib():
@@ -97,6 +98,16 @@ def _lib():
         lib.branch_attn_bwd_static.argtypes = lib.branch_attn_bwd.argtypes[:-3] + [vp]
         lib.ba_finalize_grads.restype = C.c_int
         lib.ba_finalize_grads.argtypes = [vp, vp, i64, C.c_int, vp]
+        lib.branch_attn_fwd_depth.restype = C.c_int
+        lib.branch_attn_fwd_depth.argtypes = [vp, C.c_int, vp, vp, vp, i64, i64, vp, vp, vp]
+        lib.branch_attn_bwd_depth.restype = C.c_int
+        lib.branch_attn_bwd_depth.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp,
+                                              C.c_size_t, vp]
+        lib.branch_attn_fwd_shard.restype = C.c_int
+        lib.branch_attn_fwd_shard.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, C.c_int, vp, vp, vp]
+        lib.branch_attn_bwd_shard.restype = C.c_int
+        lib.branch_attn_bwd_shard.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64,
+                                              vp, vp, vp, vp, vp, C.c_size_t, vp, C.c_int]
         lib.ba_selftest_bounded_wait.restype = C.c_int
         lib.ba_selftest_bounded_wait.argtypes = [vp, i64, vp]
         _LIB = lib
@@ -393,3 +404,106 @@ def ba_finalize_grads(src, dst=None, dtype=torch.bfloat16):
     rc = _lib().ba_finalize_grads(_p(src), _p(dst), src.numel(), code, _stream())
     _check(rc, "ba_finalize_grads")
     return dst
+
+
+# ---------------------------------------------------------------- step-major (per-depth) calls
+
+def _expect_depth(plan, q_depth, k, v):
+    p, dt, dev = plan.problem, plan.torch_dtype, plan.device
+    a = p.num_branches
+    _expect("q_depth", q_depth, (a, p.h_q, p.head_dim), dt, dev)
+    _expect("k", k, (p.rows, p.h_kv, p.head_dim), dt, dev)
+    _expect("v", v, (p.rows, p.h_kv, p.head_dim), dt, dev)
+
+
+def branch_attn_fwd_depth(plan, depth, q_depth, k, v, br_range=None, out=None, lse=None):
+    """Forward of the depth-`depth` tokens (one per branch) against the main prefix and the
+    tokens of depths <= depth of the own branch; k, v hold the branch tokens depth-major.
+    Returns (O_depth [A, h_q, D], LSE_depth [A, h_q])."""
+    p = plan.problem
+    a = p.num_branches
+    br_range = (0, a) if br_range is None else br_range
+    if out is None:
+        out = torch.empty((a, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=plan.device)
+    if lse is None:
+        lse = torch.empty((a, p.h_q), dtype=torch.float32, device=plan.device)
+    _expect_depth(plan, q_depth, k, v)
+    _expect("out", out, (a, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("lse", lse, (a, p.h_q), torch.float32, plan.device)
+    rc = _lib().branch_attn_fwd_depth(plan.handle, depth, _p(q_depth), _p(k), _p(v), br_range[0], br_range[1],
+                                      _p(out), _p(lse), _stream())
+    _check(rc, "branch_attn_fwd_depth")
+    return out, lse
+
+
+def branch_attn_bwd_depth(plan, depth, q_depth, k, v, o_depth, lse_depth, d_o_depth, dk, dv, br_range=None, dq=None):
+    """Backward of one depth: dQ_depth (input dtype) is returned, the terms of dK / dV
+    (fp32, depth-major like k, v) are added to `dk`, `dv`."""
+    p = plan.problem
+    a = p.num_branches
+    br_range = (0, a) if br_range is None else br_range
+    if dq is None:
+        dq = torch.empty((a, p.h_q, p.head_dim), dtype=plan.torch_dtype, device=plan.device)
+    _expect_depth(plan, q_depth, k, v)
+    _expect("o_depth", o_depth, (a, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("lse_depth", lse_depth, (a, p.h_q), torch.float32, plan.device)
+    _expect("d_o_depth", d_o_depth, (a, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("dq", dq, (a, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("dk", dk, (p.rows, p.h_kv, p.head_dim), torch.float32, plan.device)
+    _expect("dv", dv, (p.rows, p.h_kv, p.head_dim), torch.float32, plan.device)
+    ws = plan.workspace(OP_BWD_DEPTH)
+    rc = _lib().branch_attn_bwd_depth(plan.handle, depth, _p(q_depth), _p(k), _p(v), _p(o_depth), _p(lse_depth),
+                                      _p(d_o_depth), br_range[0], br_range[1], _p(dq), _p(dk), _p(dv),
+                                      _p(ws), ws.numel(), _stream())
+    _check(rc, "branch_attn_bwd_depth")
+    return dq
+
+
+# ---------------------------------------------------------------- ring steps on a received K/V shard
+
+def _expect_shard(plan, q_main, q_branch, k_shard, v_shard, kv_range):
+    p, dt, dev = plan.problem, plan.torch_dtype, plan.device
+    rows = kv_range[1] - kv_range[0]
+    _expect("q_main", q_main, (p.n_main, p.h_q, p.head_dim), dt, dev, optional=True)
+    _expect("q_branch", q_branch, (p.n_branch, p.h_q, p.head_dim), dt, dev, optional=p.n_branch == 0)
+    _expect("k_shard", k_shard, (rows, p.h_kv, p.head_dim), dt, dev)
+    _expect("v_shard", v_shard, (rows, p.h_kv, p.head_dim), dt, dev)
+
+
+def branch_attn_fwd_shard(plan, q_main, q_branch, k_shard, v_shard, qm_range, br_range, kv_range, acc_o, acc_lse,
+                          merge):
+    """Partial forward over the main keys [kv_range) held in (k_shard, v_shard) only;
+    writes (merge=False) or merges into (merge=True) the compact fp32 (acc_o, acc_lse)."""
+    p = plan.problem
+    t0, t1 = plan.token_range(*br_range)
+    rows = (qm_range[1] - qm_range[0]) + (t1 - t0)
+    _expect_shard(plan, q_main, q_branch, k_shard, v_shard, kv_range)
+    _expect("acc_o", acc_o, (rows, p.h_q, p.head_dim), torch.float32, plan.device)
+    _expect("acc_lse", acc_lse, (rows, p.h_q), torch.float32, plan.device)
+    rc = _lib().branch_attn_fwd_shard(plan.handle, _p(q_main), _p(q_branch), _p(k_shard), _p(v_shard),
+                                      qm_range[0], qm_range[1], br_range[0], br_range[1], kv_range[0], kv_range[1],
+                                      1 if merge else 0, _p(acc_o), _p(acc_lse), _stream())
+    _check(rc, "branch_attn_fwd_shard")
+    return acc_o, acc_lse
+
+
+def branch_attn_bwd_shard(plan, q_main, q_branch, k_shard, v_shard, o, lse, d_o, qm_range, br_range, kv_range,
+                          dq_main, dq_branch, dk_shard, dv_shard, stages=STAGE_DQ | STAGE_DKDV):
+    """Partial backward over the main keys [kv_range) held in the shard: adds to the local
+    fp32 dQ accumulators and to the shard's fp32 dK / dV accumulators."""
+    p = plan.problem
+    rows = kv_range[1] - kv_range[0]
+    _expect_shard(plan, q_main, q_branch, k_shard, v_shard, kv_range)
+    _expect("o", o, (p.rows, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("lse", lse, (p.rows, p.h_q), torch.float32, plan.device)
+    _expect("d_o", d_o, (p.rows, p.h_q, p.head_dim), plan.torch_dtype, plan.device)
+    _expect("dq_main", dq_main, (p.n_main, p.h_q, p.head_dim), torch.float32, plan.device, optional=q_main is None)
+    _expect("dq_branch", dq_branch, (p.n_branch, p.h_q, p.head_dim), torch.float32, plan.device, optional=p.n_branch == 0)
+    _expect("dk_shard", dk_shard, (rows, p.h_kv, p.head_dim), torch.float32, plan.device)
+    _expect("dv_shard", dv_shard, (rows, p.h_kv, p.head_dim), torch.float32, plan.device)
+    ws = plan.workspace(OP_BWD_FUSED if getattr(plan, "_fused_ws", False) else OP_BWD)
+    rc = _lib().branch_attn_bwd_shard(plan.handle, _p(q_main), _p(q_branch), _p(k_shard), _p(v_shard), _p(o), _p(lse),
+                                      _p(d_o), qm_range[0], qm_range[1], br_range[0], br_range[1], kv_range[0],
+                                      kv_range[1], _p(dq_main), _p(dq_branch), _p(dk_shard), _p(dv_shard),
+                                      _p(ws), ws.numel(), _stream(), stages)
+    _check(rc, "branch_attn_bwd_shard")

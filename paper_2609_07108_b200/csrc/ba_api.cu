@@ -42,6 +42,9 @@ extern "C" size_t ba_workspace_bytes(const ba_plan_t *plan, int op) {
     // delta and -LSE*log2(e), fp32, head-major [h_q, row_pitch] each
     const size_t scalars = align256((size_t)2 * plan->row_pitch * plan->prob.h_q * sizeof(float));
     if (op == BA_OP_BWD) return scalars;
+    if (op == BA_OP_BWD_DEPTH)  // plus an fp32 dQ accumulator with one row per branch
+        return scalars + align256((size_t)plan->prob.num_branches * plan->prob.h_q * plan->prob.head_dim *
+                                  sizeof(float));
     if (op == BA_OP_BWD_FUSED)  // plus the fp32 dQ accumulator of the one-kernel backward
         return scalars + align256((size_t)(plan->prob.n_main + plan->prob.n_branch) * plan->prob.h_q *
                                   plan->prob.head_dim * sizeof(float));
@@ -181,4 +184,114 @@ extern "C" int branch_attn_bwd_stages(const ba_plan_t *plan, const void *q_main,
                          dV, st, stages);
     return ba_simt_bwd(plan, r, qm, q_branch, k, v, LSE, delta, dO, accumulate, dQ_main, dQ_branch, dK, dV,
                        st, stages);
+}
+
+// ---------------------------------------------------------------- step-major (per-depth) calls
+
+static int depth_range(const ba_plan_t *plan, int depth, int64_t br_begin, int64_t br_end, BaRange *r) {
+    if (!plan) return BA_EINVAL;
+    const ba_problem_t &pr = plan->prob;
+    if (plan->impl != BA_IMPL_TC || pr.mask_kind != BA_MASK_CHAIN || pr.uniform_len <= 0) return BA_EUNSUPPORTED;
+    if (depth < 1 || depth > pr.uniform_len) return BA_EINVAL;
+    if (br_begin < 0 || br_end < br_begin || br_end > pr.num_branches) return BA_EINVAL;
+    r->qm_begin = r->qm_end = 0;
+    r->tok_begin = br_begin; r->tok_end = br_end;   // branch indices: one query row per branch
+    r->kv_begin = 0; r->kv_end = pr.n_main;
+    r->parts = BA_PART_MAIN | BA_PART_BRANCH;
+    return BA_OK;
+}
+
+extern "C" int branch_attn_fwd_depth(const ba_plan_t *plan, int depth, const void *q_depth, const void *k,
+                                     const void *v, int64_t br_begin, int64_t br_end, void *O_depth,
+                                     float *LSE_depth, void *stream) {
+    BaRange r;
+    int rc = depth_range(plan, depth, br_begin, br_end, &r);
+    if (rc != BA_OK) return rc;
+    if (br_end == br_begin) return BA_OK;
+    if (!q_depth || !k || !v || !O_depth || !LSE_depth) return BA_EINVAL;
+    return ba_tc_fwd(plan, r, nullptr, q_depth, k, v, O_depth, LSE_depth, 0, (cudaStream_t)stream, depth);
+}
+
+extern "C" int branch_attn_bwd_depth(const ba_plan_t *plan, int depth, const void *q_depth, const void *k,
+                                     const void *v, const void *O_depth, const float *LSE_depth,
+                                     const void *dO_depth, int64_t br_begin, int64_t br_end, void *dQ_depth,
+                                     float *dK, float *dV, void *workspace, size_t ws_bytes, void *stream) {
+    BaRange r;
+    int rc = depth_range(plan, depth, br_begin, br_end, &r);
+    if (rc != BA_OK) return rc;
+    if (br_end == br_begin) return BA_OK;
+    if (!q_depth || !k || !v || !O_depth || !LSE_depth || !dO_depth || !dQ_depth || !dK || !dV) return BA_EINVAL;
+    if (!workspace || ws_bytes < ba_workspace_bytes(plan, BA_OP_BWD_DEPTH) || ((uintptr_t)workspace & 255))
+        return BA_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const ba_problem_t &pr = plan->prob;
+    float *delta = (float *)workspace;
+    float *nlse2 = delta + (size_t)plan->row_pitch * pr.h_q;
+    float *acc = (float *)((char *)workspace + ba_workspace_bytes(plan, BA_OP_BWD));
+    const size_t row_elems = (size_t)pr.h_q * pr.head_dim;
+    // per-row scalars of the selected branches' depth-`depth` rows (rows are indexed by branch here)
+    if ((rc = ba_delta(O_depth, dO_depth, LSE_depth, delta, nlse2, plan->row_pitch, 0, 0, br_begin, br_end,
+                       pr.h_q, pr.head_dim, pr.dtype, st)) != BA_OK)
+        return rc;
+    BA_CUDA_CHECK(cudaMemsetAsync(acc + (size_t)br_begin * row_elems, 0,
+                                  (size_t)(br_end - br_begin) * row_elems * sizeof(float), st));
+    rc = ba_tc_bwd_fused(plan, r, nullptr, q_depth, k, v, delta, dO_depth, 1, nullptr, acc, dK, dV, st, depth);
+    if (rc != BA_OK) return rc;
+    return ba_finalize_grads(acc + (size_t)br_begin * row_elems,
+                             (__nv_bfloat16 *)dQ_depth + (size_t)br_begin * row_elems,
+                             (int64_t)((br_end - br_begin) * row_elems), pr.dtype, stream);
+}
+
+// ---------------------------------------------------------------- ring steps on a received K/V shard
+
+// The kernels address keys by their global row; a shard holds only rows [kv_begin, kv_end).
+// Tiles of 128 keys start at multiples of 128, so with both ends on such a multiple every row a
+// kernel touches lies inside the shard, and the shard can be addressed as if it were the full
+// tensor by moving its base back by kv_begin rows (no byte before the shard is ever read).
+static int shard_ok(const ba_plan_t *plan, int64_t kv_begin, int64_t kv_end) {
+    if (!plan) return BA_EINVAL;
+    if (kv_begin < 0 || kv_end < kv_begin || kv_end > plan->prob.n_main) return BA_EINVAL;
+    if ((kv_begin % 128) != 0 || ((kv_end % 128) != 0 && kv_end != plan->prob.n_main)) return BA_EINVAL;
+    return BA_OK;
+}
+
+static inline const void *rebase(const void *shard, int64_t rows_back, size_t row_bytes) {
+    return shard ? (const void *)((const char *)shard - (size_t)rows_back * row_bytes) : nullptr;
+}
+
+extern "C" int branch_attn_fwd_shard(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                                     const void *k_shard, const void *v_shard, int64_t qm_begin, int64_t qm_end,
+                                     int64_t br_begin, int64_t br_end, int64_t kv_begin, int64_t kv_end,
+                                     int merge, float *O_acc, float *LSE_acc, void *stream) {
+    int rc = shard_ok(plan, kv_begin, kv_end);
+    if (rc != BA_OK) return rc;
+    if (merge != 0 && merge != 1) return BA_EINVAL;
+    if (kv_end > kv_begin && (!k_shard || !v_shard)) return BA_EINVAL;
+    const size_t esz = plan->prob.dtype == BA_FP32 ? 4 : 2;
+    const size_t row_bytes = (size_t)plan->prob.h_kv * plan->prob.head_dim * esz;
+    const void *k = rebase(k_shard, kv_begin, row_bytes), *v = rebase(v_shard, kv_begin, row_bytes);
+    if (merge)
+        return branch_attn_fwd_partial_merge(plan, q_main, q_branch, k, v, qm_begin, qm_end, br_begin, br_end,
+                                             kv_begin, kv_end, BA_PART_MAIN, O_acc, LSE_acc, nullptr, 0, stream);
+    return branch_attn_fwd_partial(plan, q_main, q_branch, k, v, qm_begin, qm_end, br_begin, br_end, kv_begin,
+                                   kv_end, BA_PART_MAIN, O_acc, LSE_acc, nullptr, 0, stream);
+}
+
+extern "C" int branch_attn_bwd_shard(const ba_plan_t *plan, const void *q_main, const void *q_branch,
+                                     const void *k_shard, const void *v_shard, const void *O, const float *LSE,
+                                     const void *dO, int64_t qm_begin, int64_t qm_end, int64_t br_begin,
+                                     int64_t br_end, int64_t kv_begin, int64_t kv_end, float *dQ_main,
+                                     float *dQ_branch, float *dK_shard, float *dV_shard, void *workspace,
+                                     size_t ws_bytes, void *stream, int stages) {
+    int rc = shard_ok(plan, kv_begin, kv_end);
+    if (rc != BA_OK) return rc;
+    if (kv_end > kv_begin && (!k_shard || !v_shard || !dK_shard || !dV_shard)) return BA_EINVAL;
+    const size_t esz = plan->prob.dtype == BA_FP32 ? 4 : 2;
+    const size_t row_elems = (size_t)plan->prob.h_kv * plan->prob.head_dim;
+    const void *k = rebase(k_shard, kv_begin, row_elems * esz), *v = rebase(v_shard, kv_begin, row_elems * esz);
+    void *dk = (void *)rebase(dK_shard, kv_begin, row_elems * sizeof(float));
+    void *dv = (void *)rebase(dV_shard, kv_begin, row_elems * sizeof(float));
+    return branch_attn_bwd_stages(plan, q_main, q_branch, k, v, O, LSE, dO, qm_begin, qm_end, br_begin, br_end,
+                                  kv_begin, kv_end, BA_PART_MAIN, 1, dQ_main, dQ_branch, dk, dv, workspace,
+                                  ws_bytes, stream, stages);
 }

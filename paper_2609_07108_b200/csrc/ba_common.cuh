@@ -71,9 +71,11 @@ int ba_simt_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const v
                 void *dv, cudaStream_t st, int stages);
 // Tensor-core path (ba_tc_fwd.cu / ba_tc_bwd.cu)
 // partial_out: 0 = final layout in the input dtype, 1 = compact fp32, 2 = compact fp32 merged in place
+// depth > 0: step-major call (queries = the depth-`depth` tokens of branches [r.tok_begin, r.tok_end),
+// q_branch / o / lse indexed by branch, branch keys stored depth-major after the main rows)
 int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
               const void *k, const void *v, void *o, float *lse, int partial_out,
-              cudaStream_t st);
+              cudaStream_t st, int depth = 0);
 int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
               const void *k, const void *v, const float *lse, const float *delta,
               const void *d_o, int accumulate, void *dq_main, void *dq_branch, void *dk,
@@ -82,7 +84,7 @@ int ba_tc_bwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
 int ba_tc_bwd_fused(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch,
                     const void *k, const void *v, const float *delta, const void *d_o,
                     int accumulate, void *dq_main, void *dq_branch, void *dk, void *dv,
-                    cudaStream_t st);
+                    cudaStream_t st, int depth = 0);
 bool ba_tc_supported(const ba_problem_t *p);
 // Elementwise (ba_elementwise.cu)
 // Backward preprocess into head-major scratch [h_q, row_pitch]:

@@ -34,6 +34,11 @@ struct TcBwdParams {
     int has_main_q;
     int main_tiles, total_tiles;      // dQ kernel: query row tiles
     int main_key_tiles, total_key_tiles;  // dK/dV and fused kernels: key tiles
+    // Step-major (per-depth) call of the one-kernel backward: depth > 0.  Query rows are the
+    // depth-`depth` tokens of branches [r.tok_begin, r.tok_end) (branch indices), Q / dO / dQ and
+    // the per-row scalars are indexed by branch, and branch keys are stored depth-major after the
+    // main rows: token (depth j + 1, branch b) is key row N + j * num_branches + b.
+    int depth, num_branches, branch_len, branch_tiles_per_depth;
     int *status;
 };
 

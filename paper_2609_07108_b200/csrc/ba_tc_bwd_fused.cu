@@ -147,11 +147,18 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
     const int tile = (int)(blockIdx.x % p.total_key_tiles);
     const bool main_keys = tile < p.main_key_tiles;
     const int64_t n = p.meta.n_main;
-    // first key of the tile: main key index, or branch token index
+    // depth mode: branch key tile = (depth j + 1, 128 consecutive branches)
+    const int btile = tile - p.main_key_tiles;
+    const int kdepth = (p.depth && !main_keys) ? btile / p.branch_tiles_per_depth : 0;
+    // first key of the tile: main key index, or branch token index (depth mode: branch index)
     const int64_t key0 = main_keys ? p.r.kv_begin + (int64_t)tile * kTile
-                                   : p.r.tok_begin + (int64_t)(tile - p.main_key_tiles) * kTile;
+                         : p.depth ? p.r.tok_begin + (int64_t)(btile % p.branch_tiles_per_depth) * kTile
+                                   : p.r.tok_begin + (int64_t)btile * kTile;
     const int64_t key_end = main_keys ? p.r.kv_end : p.r.tok_end;
-    const int64_t gkey0 = main_keys ? key0 : n + key0;
+    const int64_t gkey0 = main_keys ? key0 : p.depth ? n + (int64_t)kdepth * p.num_branches + key0 : n + key0;
+    // global row number of branch query 0 (rows of dO and of the per-row scalars): branch rows
+    // follow the main rows, except in depth mode, where those tensors hold one row per branch
+    const int64_t qbase = p.depth ? 0 : n;
 
     if (tid == 0) {
         mbar_init(&sm.kv_full, 1);
@@ -186,6 +193,13 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                 my_qend = p.meta.key_qend[kk];
                 my_bq0 = p.meta.key_bq_begin[kk];
                 my_bq1 = p.meta.key_bq_end[kk];
+                if (p.depth) {   // token ranges -> branch ranges (every branch has branch_len tokens)
+                    my_bq0 /= p.branch_len;
+                    my_bq1 /= p.branch_len;
+                }
+            } else if (p.depth) {
+                my_bq0 = (int)kk;          // seen by the query of its own branch only
+                my_bq1 = (int)kk + 1;
             } else {
                 my_bq0 = p.meta.br_start[kk];
                 my_bq1 = p.meta.br_end[kk];
@@ -217,7 +231,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
         b1 = min((int64_t)sm.bq1_max, p.r.tok_end);
     }
     const int64_t ma = m0 & ~(int64_t)3;
-    const int64_t ba = ((n + b0) & ~(int64_t)3) - n;   // may be as low as -3
+    const int64_t ba = ((qbase + b0) & ~(int64_t)3) - qbase;   // may be as low as -3
     const int n_sub_main = m1 > m0 ? (int)((m1 - ma + kTile - 1) / kTile) : 0;
     const int n_sub_br = b1 > b0 ? (int)((b1 - ba + kTile - 1) / kTile) : 0;
     const int n_sub = n_sub_main + n_sub_br;
@@ -254,7 +268,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                 const int u = n_sub - 1 - s;   // tiles are walked from the last one down (see n_iter)
                 const bool seg_main = u < n_sub_main;
                 const int64_t r0 = seg_main ? ma + (int64_t)u * kTile : ba + (int64_t)(u - n_sub_main) * kTile;
-                const int64_t grow0 = seg_main ? r0 : n + r0;
+                const int64_t grow0 = seg_main ? r0 : qbase + r0;
                 const CUtensorMap *tq = seg_main ? &tm_q_main : &tm_q_branch;
                 mbar_expect_tx(&sm.q_full[st], 2 * kTileBytes + 2 * kTile * 4);
                 for (int half = 0; half < 2; ++half) {
@@ -270,7 +284,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                     const int u2 = n_sub - 1 - ps;
                     const bool main2 = u2 < n_sub_main;
                     const int64_t r2 = main2 ? ma + (int64_t)u2 * kTile : ba + (int64_t)(u2 - n_sub_main) * kTile;
-                    const int64_t g2 = main2 ? r2 : n + r2;
+                    const int64_t g2 = main2 ? r2 : qbase + r2;
                     const CUtensorMap *tq2 = main2 ? &tm_q_main : &tm_q_branch;
                     for (int half = 0; half < 2; ++half) {
                         tma_prefetch_3d(tq2, half * 64, h2, (int)r2);
@@ -473,6 +487,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
                         vis = bit_range(max(my_key, rbeg) - r0h, min(my_qend, rend) - 1 - r0h);
                     else           // branch tokens anchored at or after the key, inside its sequence
                         vis = bit_range(max(my_bq0, rbeg) - r0h, min(my_bq1, rend) - 1 - r0h);
+                } else if (p.depth) {
+                    // my key is token (kdepth + 1) of branch my_key: seen by that branch's query
+                    if (my_key >= rbeg && my_key < rend) vis = bit_range(my_key - r0h, my_key - r0h);
                 } else {
                     // own-branch tokens whose mask has my bit (few, short tiles)
                     const int lo_c = max(max(my_bq0, rbeg) - r0h, 0);
@@ -579,7 +596,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_
 
 int ba_tc_bwd_fused(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
                     const void *v, const float *delta, const void *d_o, int accumulate, void *dq_main,
-                    void *dq_branch, void *dk, void *dv, cudaStream_t st) {
+                    void *dq_branch, void *dk, void *dv, cudaStream_t st, int depth) {
     // dq_main / dq_branch are always fp32 accumulators (summed with atomic adds);
     // `accumulate` says whether dK / dV are fp32 accumulators too or written in bf16
     // the dynamic shared-memory limit is a per-device attribute of the kernel
@@ -617,20 +634,29 @@ int ba_tc_bwd_fused(const ba_plan *pl, const BaRange &r, const void *q_main, con
     p.has_main_q = q_main != nullptr;
     p.status = pl->dev_status;
     const int64_t kmt = (r.parts & BA_PART_MAIN) ? (r.kv_end - r.kv_begin + kTile - 1) / kTile : 0;
-    const int64_t kbt = (r.parts & BA_PART_BRANCH) ? (r.tok_end - r.tok_begin + kTile - 1) / kTile : 0;
+    int64_t kbt = (r.parts & BA_PART_BRANCH) ? (r.tok_end - r.tok_begin + kTile - 1) / kTile : 0;
+    p.depth = depth;
+    p.num_branches = pr.num_branches;
+    p.branch_len = pr.uniform_len;
+    p.branch_tiles_per_depth = (int)kbt;
+    if (depth) kbt *= depth;    // the tokens of depths 1 .. depth of the selected branches are keys
     p.main_key_tiles = (int)kmt;
     p.total_key_tiles = (int)(kmt + kbt);
     if (p.total_key_tiles == 0) return BA_OK;
 
     CUtensorMap tq_main, tq_branch, tgo, tk, tv;
+    // depth mode: key rows of depths <= depth only (later rows read as zero); dO holds one row per branch
     const uint64_t all_rows = (uint64_t)(pr.n_main + pr.n_branch);
-    if (!make_tmap_rhd(&tk, k, all_rows, pr.h_kv, 128, kTile) || !make_tmap_rhd(&tv, v, all_rows, pr.h_kv, 128, kTile) ||
-        !make_tmap_rhd(&tgo, d_o, all_rows, pr.h_q, 128, kTile))
+    const uint64_t kv_rows = depth ? (uint64_t)(pr.n_main + (int64_t)depth * pr.num_branches) : all_rows;
+    const uint64_t go_rows = depth ? (uint64_t)pr.num_branches : all_rows;
+    if (!make_tmap_rhd(&tk, k, kv_rows, pr.h_kv, 128, kTile) || !make_tmap_rhd(&tv, v, kv_rows, pr.h_kv, 128, kTile) ||
+        !make_tmap_rhd(&tgo, d_o, go_rows, pr.h_q, 128, kTile))
         return BA_EINVAL;
     const void *qm = q_main ? q_main : q_branch;
     const void *qb = (q_branch && pr.n_branch > 0) ? q_branch : q_main;
-    const uint64_t qm_rows = q_main ? (uint64_t)pr.n_main : (uint64_t)pr.n_branch;
-    const uint64_t qb_rows = (q_branch && pr.n_branch > 0) ? (uint64_t)pr.n_branch : (uint64_t)pr.n_main;
+    const uint64_t qm_rows = depth ? (uint64_t)pr.num_branches : q_main ? (uint64_t)pr.n_main : (uint64_t)pr.n_branch;
+    uint64_t qb_rows = (q_branch && pr.n_branch > 0) ? (uint64_t)pr.n_branch : (uint64_t)pr.n_main;
+    if (depth) qb_rows = (uint64_t)pr.num_branches;
     if (!make_tmap_rhd(&tq_main, qm, qm_rows, pr.h_q, 128, kTile) ||
         !make_tmap_rhd(&tq_branch, qb, qb_rows, pr.h_q, 128, kTile))
         return BA_EINVAL;

@@ -55,6 +55,11 @@ struct TcFwdParams {
     float scale_log2;
     int partial_out;
     int main_tiles, total_tiles;
+    // Step-major (per-depth) call: depth > 0.  The query rows are the depth-`depth` tokens of
+    // branches [tok_begin, tok_end) (r.tok_* hold BRANCH indices then), the query tensor and the
+    // outputs are indexed by branch, and the branch keys are stored depth-major after the main
+    // rows: token (depth j + 1, branch b) is key row N + j * num_branches + b.
+    int depth, num_branches, branch_len;
     int *status;
 };
 
@@ -202,13 +207,14 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
         my_row = row0 + (tid & 127);
         valid = my_row < row_end;
         if (valid) {
-            const int64_t grow = is_main ? my_row : n + my_row;
+            // depth mode: my_row is a branch index; all tokens of a branch share the causal prefix
+            const int64_t grow = is_main ? my_row : n + (p.depth ? my_row * p.branch_len : my_row);
             if (p.r.parts & BA_PART_MAIN) {
                 lo = max(p.meta.row_lo[grow], (int)p.r.kv_begin);
                 hi = min(p.meta.row_hi[grow], (int)p.r.kv_end - 1);
                 if (hi < lo) { lo = 1; hi = 0; }
             }
-            if (!is_main && (p.r.parts & BA_PART_BRANCH)) {
+            if (!is_main && (p.r.parts & BA_PART_BRANCH) && !p.depth) {
                 bstart = p.meta.br_start[my_row];
                 bmask = p.meta.br_mask[my_row];
             }
@@ -219,7 +225,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 } else {
                     atomicMax(&sm.lo_max, INT_MAX); atomicMin(&sm.hi_min, -1);
                 }
-                if (!is_main && (p.r.parts & BA_PART_BRANCH)) {
+                if (!is_main && (p.r.parts & BA_PART_BRANCH) && !p.depth) {
                     atomicMin(&sm.bs_min, bstart);
                     atomicMax(&sm.be_max, p.meta.br_end[my_row]);
                 }
@@ -240,6 +246,9 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
     }
     const int bs = sm.bs_min;
     if (sm.be_max > bs) n_br = (sm.be_max - bs + kTile - 1) / kTile;
+    // depth mode: one key tile per depth 1 .. depth, holding the tokens of this tile's own branches
+    // in branch order, so row i sees exactly column i of each of them
+    if (p.depth && (p.r.parts & BA_PART_BRANCH)) n_br = p.depth;
     const int T = n_main_tiles + n_br;
     const int full_lo = sm.lo_max, full_hi = sm.hi_min;
 
@@ -259,7 +268,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                 if (it >= kStages) ok = mbar_wait(&sm.kv_empty[s], ((it / kStages) - 1) & 1, abort_flag);
                 if (!ok) break;
                 const int krow = j < n_main_tiles ? (kt0 + j) * kTile
-                                                  : (int)n + bs + (j - n_main_tiles) * kTile;
+                                 : p.depth ? (int)n + (j - n_main_tiles) * p.num_branches + (int)row0
+                                           : (int)n + bs + (j - n_main_tiles) * kTile;
                 const CUtensorMap *tkv = (it & 1) ? &tm_v : &tm_k;
                 mbar_expect_tx(&sm.kv_full[s], kTileBytes);
                 tma_load_3d(sm.kv[s], tkv, 0, g, krow, &sm.kv_full[s]);
@@ -358,6 +368,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
                     vis[0] = bit_range(lo - kj, hi - kj);
                     vis[1] = bit_range(lo - kj - 64, hi - kj - 64);
                 }
+            } else if (p.depth) {
+                masked = true;
+                const int c = tid & 127;     // depth mode: column c is the same branch as row c
+                vis[0] = (valid && c < 64) ? 1ull << c : 0ull;
+                vis[1] = (valid && c >= 64) ? 1ull << (c - 64) : 0ull;
             } else {
                 masked = true;
                 // column c is branch token bs + 128 (j - n_main_tiles) + c; bit c = bmask bit (c + off)
@@ -466,7 +481,8 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q_main, const __grid_consta
             const bool do_store = ok && valid && (i == 0 || second_head);
             const int h = i == 0 ? h0 : h1;
             int64_t orow = is_main ? my_row : n + my_row;
-            if (p.partial_out)
+            if (p.depth) orow = my_row;              // outputs of a per-depth call are indexed by branch
+            else if (p.partial_out)
                 orow = is_main ? my_row - p.r.qm_begin : (p.r.qm_end - p.r.qm_begin) + (my_row - p.r.tok_begin);
             const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
             const size_t base = ((size_t)orow * p.h_q + h) * 128;
@@ -521,7 +537,7 @@ bool ba_tc_supported(const ba_problem_t *p) {
 }
 
 int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const void *q_branch, const void *k,
-              const void *v, void *o, float *lse, int partial_out, cudaStream_t st) {
+              const void *v, void *o, float *lse, int partial_out, cudaStream_t st, int depth) {
     // the dynamic shared-memory limit is a per-device attribute of the kernel
     static bool attr_set[64] = {};
     int dev = 0;
@@ -546,6 +562,9 @@ int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
     p.scale_log2 = pl->scale * kLog2e;
     p.partial_out = partial_out;   // 0 final layout, 1 compact fp32, 2 compact fp32 merged in place
     p.status = pl->dev_status;
+    p.depth = depth;
+    p.num_branches = pr.num_branches;
+    p.branch_len = pr.uniform_len;
     const int64_t mt = q_main ? (r.qm_end - r.qm_begin + kTile - 1) / kTile : 0;
     const int64_t bt = (r.tok_end - r.tok_begin + kTile - 1) / kTile;
     p.main_tiles = (int)mt;
@@ -553,14 +572,17 @@ int ba_tc_fwd(const ba_plan *pl, const BaRange &r, const void *q_main, const voi
     if (p.total_tiles == 0) return BA_OK;
 
     CUtensorMap tq_main, tq_branch, tk, tv;
-    const uint64_t kv_rows = (uint64_t)(pr.n_main + pr.n_branch);
+    // depth mode: only the key rows of depths <= depth exist yet; rows beyond them read as zero
+    const uint64_t kv_rows = depth ? (uint64_t)(pr.n_main + (int64_t)depth * pr.num_branches)
+                                   : (uint64_t)(pr.n_main + pr.n_branch);
     if (!make_tmap_rhd(&tk, k, kv_rows, pr.h_kv, 128, kTile) || !make_tmap_rhd(&tv, v, kv_rows, pr.h_kv, 128, kTile))
         return BA_EINVAL;
     // an absent query tensor still needs a valid map object: alias the other one
     const void *qm = q_main ? q_main : q_branch;
     const void *qb = (q_branch && pr.n_branch > 0) ? q_branch : q_main;
-    const uint64_t qm_rows = q_main ? (uint64_t)pr.n_main : (uint64_t)pr.n_branch;
-    const uint64_t qb_rows = (q_branch && pr.n_branch > 0) ? (uint64_t)pr.n_branch : (uint64_t)pr.n_main;
+    const uint64_t qm_rows = depth ? (uint64_t)pr.num_branches : q_main ? (uint64_t)pr.n_main : (uint64_t)pr.n_branch;
+    uint64_t qb_rows = (q_branch && pr.n_branch > 0) ? (uint64_t)pr.n_branch : (uint64_t)pr.n_main;
+    if (depth) qb_rows = (uint64_t)pr.num_branches;     // the queries of one depth: one row per branch
     if (!make_tmap_rhd(&tq_main, qm, qm_rows, pr.h_q, 128, kTile) ||
         !make_tmap_rhd(&tq_branch, qb, qb_rows, pr.h_q, 128, kTile))
         return BA_EINVAL;
