@@ -40,12 +40,12 @@ def test_taps_cross_processes_through_the_mailbox(tmp_path):
             dims = {DIMS!r}
             srcs = [tap.Source({name!r}, s, ipc_handle=handle) for s in range(len(dims))]
             stream = torch.cuda.current_stream().cuda_stream
-            keep = []
+            taps = {{(m, s): torch.full(({N_ROWS}, d), float(s + 1) + m / 16.0, dtype=torch.bfloat16, device="cuda")
+                    for m in range(1, {N_MICRO} + 1) for s, d in enumerate(dims)}}
+            torch.cuda.synchronize()
             for m in range(1, {N_MICRO} + 1):
                 for s, d in enumerate(dims):
-                    taps = torch.full(({N_ROWS}, d), float(s + 1) + m / 16.0, dtype=torch.bfloat16, device="cuda")
-                    srcs[s].send(taps, m, stream, 60.0)   # waits (bounded) until the draft has read microbatch m - 1
-                    keep.append(taps)
+                    srcs[s].send(taps[(m, s)], m, stream, 60.0)   # waits (bounded) until the draft has read microbatch m - 1
             torch.cuda.synchronize()
             for x in srcs:
                 x.close()
@@ -59,7 +59,7 @@ def test_taps_cross_processes_through_the_mailbox(tmp_path):
                 t0 = t0 or time.perf_counter()
                 assert nbytes == N_ROWS * d * 2
                 view = mb.slot_tensor(s, nbytes).view(torch.bfloat16)
-                bad = (view.float() != pattern(s, m)).sum()          # the draft's read of the slot, on its stream
+                bad = torch.count_nonzero(view != pattern(s, m))       # the draft's read of the slot, on its stream
                 mb.release(s, m, stream)                             # handed back once that read has run
                 assert int(bad.item()) == 0, (s, m)
                 total += nbytes
