@@ -692,7 +692,10 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     main = torch.cuda.current_stream()
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     fused = use_fused_bwd(args, p, plan, ba)
-    for _ in range(steps):
+    streamed = bool(cp) and backward and full and t.get("_mode", "zigzag") == "zigzag"
+    for _ in range(steps if streamed else 0):
+        e2e_step_streamed(torch, rec, plan, p, t, cp, fused, host_in, host_out, main, s_in, s_out)
+    for _ in range(0 if streamed else steps):
         for k in names:
             if k != "d_o":
                 h2d_copy(t[k], k)
@@ -729,7 +732,75 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     value, _ = aggregate_throughput(dist, flops * steps, ms, device)
     return {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "steps": steps, "ms_per_step": round(ms / steps, 3),
-            "host_buffers": "pinned, full size" if full else "pinned 1 GiB staging (host memory too small for full copies)"}
+            "host_buffers": "pinned, full size" if full else "pinned 1 GiB staging (host memory too small for full copies)",
+            "copies": ("streamed per query chunk: K, V, then the query rows in the order the chunks are used, dO behind "
+                       "the forward; O / LSE and each chunk's dQ behind the backward, dK / dV at the end") if streamed
+                      else "whole tensors: Q, K, V before the forward, dO behind it; O / LSE behind the backward, gradients after it"}
+
+
+def e2e_step_streamed(torch, rec, plan, p, t, cp, fused, host_in, host_out, main, s_in, s_out):
+    """One end-to-end step of the zigzag workload with the host copies streamed chunk by chunk:
+    the forward of a query chunk starts as soon as K, V and that chunk's query rows are on the
+    device, and a chunk's dQ leaves for the host as soon as its last backward block is done."""
+    from paper_2609_07108_b200 import zigzag
+    n = p.n_main
+    bounds = zigzag.chunk_bounds(n, cp)
+    anchors = np.asarray(p.anchor_idx, dtype=np.int64)
+    ws = t["_ws"]
+
+    class Hooks:
+        q_events = {}
+
+        @staticmethod
+        def q_ready(qc):
+            main.wait_event(Hooks.q_events[qc])
+
+        @staticmethod
+        def dq_done(qc, qm, tok):
+            ev = torch.cuda.Event()
+            ev.record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev)
+                host_out[2][qm[0]:qm[1]].copy_(ws.outs[0][qm[0]:qm[1]], non_blocking=True)
+                host_out[3][tok[0]:tok[1]].copy_(ws.outs[1][tok[0]:tok[1]], non_blocking=True)
+
+    start = torch.cuda.Event()
+    start.record(main)
+    with torch.cuda.stream(s_in):
+        s_in.wait_event(start)
+        t["k"].copy_(host_in["k"], non_blocking=True)
+        t["v"].copy_(host_in["v"], non_blocking=True)
+        for qc in zigzag.chunk_order(cp):
+            q0, q1 = bounds[qc]
+            b0 = int(np.searchsorted(anchors, q0, side="left"))
+            b1 = int(np.searchsorted(anchors, q1, side="left"))
+            t0, t1 = plan.token_range(b0, b1)
+            t["q_main"][q0:q1].copy_(host_in["q_main"][q0:q1], non_blocking=True)
+            t["q_branch"][t0:t1].copy_(host_in["q_branch"][t0:t1], non_blocking=True)
+            ev = torch.cuda.Event()
+            ev.record(s_in)
+            Hooks.q_events[qc] = ev
+        t["d_o"].copy_(host_in["d_o"], non_blocking=True)
+        go_in = torch.cuda.Event()
+        go_in.record(s_in)
+    o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp, out=t.get("_o"),
+                               lse=t.get("_lse"), ws=ws, hooks=Hooks)
+    fwd_done = torch.cuda.Event()
+    fwd_done.record(main)
+    with torch.cuda.stream(s_out):
+        s_out.wait_event(fwd_done)
+        host_out[0].copy_(o, non_blocking=True)
+        host_out[1].copy_(lse, non_blocking=True)
+    main.wait_event(go_in)
+    grads = zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp, fused=fused,
+                            ws=ws, hooks=Hooks)
+    done = torch.cuda.Event()
+    done.record(main)
+    with torch.cuda.stream(s_out):
+        s_out.wait_event(done)
+        host_out[4].copy_(grads[2], non_blocking=True)
+        host_out[5].copy_(grads[3], non_blocking=True)
+    main.wait_stream(s_out)
 
 
 # ----------------------------------------------------------------------------

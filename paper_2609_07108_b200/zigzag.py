@@ -122,10 +122,17 @@ class Workspace:
             self.outs = tuple(torch.empty(s, dtype=plan.torch_dtype, device=dev) for s in shapes)
 
 
-def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None, ws=None):
+def chunk_order(cp: int) -> List[int]:
+    """Query chunks in the order the drivers work through them (rank by rank)."""
+    return [qc for rank in range(cp) for qc in rank_chunks(rank, cp)]
+
+
+def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None, ws=None, hooks=None):
     """Emulated CP forward: per (rank, step) partial calls, each merged into the
     running (O, LSE) by Eq. (lse-merge) -- in the kernel's epilogue on tensor-core
     plans, by `lse_merge` otherwise.  `out` may be fp32 (no rounding of O).
+    `hooks.q_ready(qc)`, if given, is called before the first call that reads the
+    query rows of chunk qc (a caller that streams the queries in waits there).
     Returns (O [N+M,h_q,D], LSE fp32, number of library launches)."""
     import torch
     p = plan.problem
@@ -147,6 +154,8 @@ def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None, ws=None):
     for rank in range(cp):
         for qc in rank_chunks(rank, cp):
             mine = [b for b in blocks if b.rank == rank and b.q_chunk == qc]
+            if hooks is not None:
+                hooks.q_ready(qc)
             t0, t1 = plan.token_range(*mine[0].br)
             rows = csize + t1 - t0
             a_o, a_l = acc_o[:rows], acc_l[:rows]
@@ -176,13 +185,17 @@ def forward(ba, plan, q_main, q_branch, k, v, cp, out=None, lse=None, ws=None):
     return out, lse, launches
 
 
-def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp, fused=False, ws=None):
+def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp, fused=False, ws=None, hooks=None):
     """Emulated CP backward: the same (rank, step) blocks, gradients accumulated
     in fp32 and converted once at the end.  Returns (dQ_main, dQ_branch, dK, dV,
     launches) in the input dtype.  `fused`: one kernel per block for dQ, dK and
     dV (dQ summed with atomic adds) instead of a dQ and a dK/dV kernel.
     The per-row scalars (delta and -LSE log2 e) of a query chunk are prepared once,
-    before the chunk's first block, not once per block."""
+    before the chunk's first block, not once per block.  dQ of a query chunk is
+    complete when the chunk's last block is done (as on the rank that owns it) and is
+    converted right then; `hooks.dq_done(qc, (q0, q1), (t0, t1))`, if given, is called
+    after that (a caller that streams the gradients out starts there).  dK and dV
+    are complete, and converted, at the end."""
     p = plan.problem
     if ws is None or ws.grads is None:
         ws = Workspace(ba, plan, cp, backward=True)
@@ -208,5 +221,15 @@ def backward(ba, plan, q_main, q_branch, k, v, o, lse, d_o, cp, fused=False, ws=
                     ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, stages=ba.STAGE_DQ, **rng, **common)
                     ba.branch_attn_bwd(plan, q_main, q_branch, k, v, o, lse, d_o, stages=ba.STAGE_DKDV, **rng, **common)
                     launches += 2
-    outs = tuple(ba.ba_finalize_grads(g, dst=d) for g, d in zip(grads, ws.outs))
-    return (*outs, launches + 4)
+            q0, q1 = mine[0].qm
+            t0, t1 = plan.token_range(*mine[0].br)
+            ba.ba_finalize_grads(grads[0][q0:q1], dst=ws.outs[0][q0:q1])
+            launches += 1
+            if t1 > t0:
+                ba.ba_finalize_grads(grads[1][t0:t1], dst=ws.outs[1][t0:t1])
+                launches += 1
+            if hooks is not None:
+                hooks.dq_done(qc, (q0, q1), (t0, t1))
+    ba.ba_finalize_grads(grads[2], dst=ws.outs[2])
+    ba.ba_finalize_grads(grads[3], dst=ws.outs[3])
+    return (*ws.outs, launches + 2)
