@@ -631,7 +631,10 @@ def run_ours(args):
 def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     """Same step, inputs in pinned host memory: H2D of Q/K/V/dO, the library
     calls, D2H of O/LSE and the gradients, all inside the timed region.  The copy
-    of dO overlaps the forward, the copy of O and LSE overlaps the backward."""
+    of dO overlaps the forward, the copy of O and LSE overlaps the backward; on the
+    zigzag workload the query rows also arrive, and dQ also leaves, chunk by chunk
+    (`e2e_step_streamed`), so that only K, V and the first chunk are waited for
+    before the first kernel and only dK, dV and the last chunk's dQ after the last."""
     import psutil
     names = tuple(k for k in ("q_main", "q_branch", "k", "v") + (("d_o",) if backward else ()) if t[k] is not None)
     h2d = sum(t[k].numel() * t[k].element_size() for k in names)
@@ -684,17 +687,19 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     if dist is not None:
         dist.barrier()
     steps = max(1, min(args.steps, args.e2e_steps))
-    s_ev = torch.cuda.Event(enable_timing=True)
-    e_ev = torch.cuda.Event(enable_timing=True)
-    s_ev.record()
     # The cotangent is only needed by the backward and O / LSE are final after the
     # forward: their copies run on side streams behind the forward / the backward.
     main = torch.cuda.current_stream()
-    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()     # long-lived objects: made once, outside the steps
     fused = use_fused_bwd(args, p, plan, ba)
+    s_ev = torch.cuda.Event(enable_timing=True)
+    e_ev = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s_ev.record()
     streamed = bool(cp) and backward and full and t.get("_mode", "zigzag") == "zigzag"
+    marks = []
     for _ in range(steps if streamed else 0):
-        e2e_step_streamed(torch, rec, plan, p, t, cp, fused, host_in, host_out, main, s_in, s_out)
+        marks = e2e_step_streamed(torch, rec, plan, p, t, cp, fused, host_in, host_out, main, s_in, s_out)
     for _ in range(0 if streamed else steps):
         for k in names:
             if k != "d_o":
@@ -730,7 +735,11 @@ def run_e2e(torch, ba, plan, p, t, cp, backward, flops, dist, device, args):
     torch.cuda.synchronize()
     ms = s_ev.elapsed_time(e_ev)
     value, _ = aggregate_throughput(dist, flops * steps, ms, device)
-    return {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+    timeline = None
+    if marks:   # last step: when its phases ended, in ms after the step's start
+        timeline = {name: round(marks[0][1].elapsed_time(ev), 1) for name, ev in marks[1:]}
+        timeline["step_start_in_timed_region"] = round(s_ev.elapsed_time(marks[0][1]), 1)
+    return {"timeline_ms": timeline, "value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "steps": steps, "ms_per_step": round(ms / steps, 3),
             "host_buffers": "pinned, full size" if full else "pinned 1 GiB staging (host memory too small for full copies)",
             "copies": ("streamed per query chunk: K, V, then the query rows in the order the chunks are used, dO behind "
@@ -764,12 +773,19 @@ def e2e_step_streamed(torch, rec, plan, p, t, cp, fused, host_in, host_out, main
                 host_out[2][qm[0]:qm[1]].copy_(ws.outs[0][qm[0]:qm[1]], non_blocking=True)
                 host_out[3][tok[0]:tok[1]].copy_(ws.outs[1][tok[0]:tok[1]], non_blocking=True)
 
-    start = torch.cuda.Event()
-    start.record(main)
+    def mark(name, stream=main):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream)
+        marks.append((name, ev))
+        return ev
+
+    marks = []
+    start = mark("start")
     with torch.cuda.stream(s_in):
         s_in.wait_event(start)
         t["k"].copy_(host_in["k"], non_blocking=True)
         t["v"].copy_(host_in["v"], non_blocking=True)
+        mark("k_v_on_device", s_in)
         for qc in zigzag.chunk_order(cp):
             q0, q1 = bounds[qc]
             b0 = int(np.searchsorted(anchors, q0, side="left"))
@@ -780,27 +796,29 @@ def e2e_step_streamed(torch, rec, plan, p, t, cp, fused, host_in, host_out, main
             ev = torch.cuda.Event()
             ev.record(s_in)
             Hooks.q_events[qc] = ev
+        mark("queries_on_device", s_in)
         t["d_o"].copy_(host_in["d_o"], non_blocking=True)
-        go_in = torch.cuda.Event()
-        go_in.record(s_in)
+        go_in = mark("cotangent_on_device", s_in)
     o, lse, _ = zigzag.forward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], cp, out=t.get("_o"),
                                lse=t.get("_lse"), ws=ws, hooks=Hooks)
-    fwd_done = torch.cuda.Event()
-    fwd_done.record(main)
+    fwd_done = mark("forward_done")
     with torch.cuda.stream(s_out):
         s_out.wait_event(fwd_done)
         host_out[0].copy_(o, non_blocking=True)
         host_out[1].copy_(lse, non_blocking=True)
+        mark("o_lse_on_host", s_out)
     main.wait_event(go_in)
     grads = zigzag.backward(rec, plan, t["q_main"], t["q_branch"], t["k"], t["v"], o, lse, t["d_o"], cp, fused=fused,
                             ws=ws, hooks=Hooks)
-    done = torch.cuda.Event()
-    done.record(main)
+    done = mark("backward_done")
     with torch.cuda.stream(s_out):
         s_out.wait_event(done)
+        mark("dq_on_host", s_out)
         host_out[4].copy_(grads[2], non_blocking=True)
         host_out[5].copy_(grads[3], non_blocking=True)
     main.wait_stream(s_out)
+    mark("gradients_on_host")
+    return marks
 
 
 # ----------------------------------------------------------------------------
