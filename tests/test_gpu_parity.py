@@ -175,6 +175,37 @@ def test_bounded_wait_runs_out_and_the_library_carries_on(ba, oracle):
     check_full(ba, oracle, p, seed=3, std=0.5, impl=ba.IMPL_TC)                        # the context is intact
 
 
+def test_binding_refuses_tensors_the_kernels_could_not_address(ba):
+    """The library sees raw pointers: a strided view, a wrong dtype, shape or device must be
+    stopped in the binding, before any kernel could read or write outside an allocation."""
+    p = W.odd_shapes(W.CHAIN, head_dim=128, dtype="bf16")
+    d = to_dev(p, W.make_tensors(p, seed=2, std=0.5))
+    plan = ba.Plan(p, impl=ba.IMPL_TC)
+    o, lse = ba.branch_attn_fwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"])
+    wide = torch.zeros((p.rows, 2 * p.h_kv, p.head_dim), dtype=torch.bfloat16, device="cuda")
+    cases = [
+        dict(k=wide[:, ::2]),                                   # strided view of the right shape
+        dict(k=d["k"].float()),                                 # wrong dtype
+        dict(k=d["k"][:-1]),                                    # one row short
+        dict(q_branch=d["q_branch"].cpu()),                     # wrong device
+        dict(v=None),                                           # missing
+    ]
+    for bad in cases:
+        args = dict(q_main=d["q_main"], q_branch=d["q_branch"], k=d["k"], v=d["v"])
+        args.update(bad)
+        with pytest.raises(ValueError):
+            ba.branch_attn_fwd(plan, args["q_main"], args["q_branch"], args["k"], args["v"])
+        with pytest.raises(ValueError):
+            ba.branch_attn_bwd(plan, args["q_main"], args["q_branch"], args["k"], args["v"], o, lse, d["d_o"])
+    with pytest.raises(ValueError):                              # outputs are checked too
+        ba.branch_attn_fwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"], out=o[:, :, :64])
+    with pytest.raises(ValueError):
+        ba.branch_attn_bwd(plan, d["q_main"], d["q_branch"], d["k"], d["v"], o, lse[:, :2], d["d_o"])
+    with pytest.raises(ValueError):
+        ba.ba_finalize_grads(torch.zeros((4, 8), device="cuda")[:, ::2])
+    plan.check()
+
+
 # --------------------------------------------------------------------- merge
 
 def test_lse_merge_matches_oracle(ba, oracle):
